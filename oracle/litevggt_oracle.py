@@ -1,0 +1,319 @@
+"""CPU oracle for geometry-aware cached token merging around VGGT's global attention.
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow float64 numpy restatement of what the
+paper defines (Sec. 3.4 "Geometry-aware Cached Token Merging", Sec. 3.1 for the token
+layout and the global attention layer).  It shares no code with the CUDA library and
+must never be imported by it: only the test-suite, the smoke check and the benchmark's
+CPU-baseline leg may call it.
+
+Conventions
+  * F frames; patch grid gh x gw; P = gh*gw patch tokens and S special tokens per
+    frame (1 camera + 4 register, Sec. 3.1); T = P + S; N = F*T tokens; D channels.
+  * token index i = f*T + t; t < S are the special tokens, t = S + py*gw + px patches.
+  * inputs arrive as the same bf16 values the GPU sees, widened to float64; nothing in
+    here rounds to a narrower type.
+  * every tie is broken towards the lowest index.
+
+Where the paper leaves a choice open (normalisation, window, padding, the merge-ratio
+knob, odd grids ...) the reading taken is stated in the function's docstring.
+
+Parity status: every function below is pinned by tests against closed forms,
+invariants, library routines on special cases or brute force; the path as a whole is
+"parity unpinned" against the authors' own implementation, which is not available.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+CLS_PROTECTED = 0  # special tokens (never merged, never anchors)
+CLS_GA = 1         # top geometric-importance tokens, excluded from merging
+CLS_DST = 2        # anchors
+CLS_SRC = 3        # merge candidates
+
+
+# --------------------------------------------------------------------------------------
+# sizes
+# --------------------------------------------------------------------------------------
+def derived_sizes(frames, grid_h, grid_w, n_special=5, merge_ratio=0.5, ga_keep_frac=0.10,
+                  cell_h=2, cell_w=2):
+    """Token counts that follow from the partition rules of Sec. 3.4 ("GA Token
+    Partitioning").  Per non-first frame: one anchor per (clipped) cell, floor(frac*P)
+    GA tokens, the rest are src.  First frame: all P patches are anchors.  The
+    merge-ratio knob (not in the paper; the paper merges every src) removes
+    R = min(|Src|, floor(r*N)) tokens."""
+    p = grid_h * grid_w
+    t = p + n_special
+    n = frames * t
+    n_dst_f = -(-grid_h // cell_h) * -(-grid_w // cell_w)
+    n_ga_f = int(np.floor(ga_keep_frac * p + 1e-9))
+    n_ga_f = min(n_ga_f, p - n_dst_f)
+    n_src_f = p - n_dst_f - n_ga_f
+    n_src = (frames - 1) * n_src_f
+    n_dst = p + (frames - 1) * n_dst_f
+    r = min(n_src, int(np.floor(merge_ratio * n + 1e-9)))
+    return dict(P=p, T=t, N=n, n_dst_frame=n_dst_f, n_ga_frame=n_ga_f, n_src_frame=n_src_f,
+                n_src=n_src, n_dst=n_dst, R=r, M=n - r)
+
+
+# --------------------------------------------------------------------------------------
+# step 1: geometry-aware map
+# --------------------------------------------------------------------------------------
+def grad_map(images, patch_px=14):
+    """Grad map Psi_g (Sec. 3.4, "Pixel Gradient"): Sobel operator on image intensity,
+    downsampled to token granularity.
+
+    Reading: intensity = mean of R,G,B; 3x3 Sobel pair, replicate padding at the image
+    border; magnitude sqrt(gx^2+gy^2); average over each patch_px x patch_px patch.
+    images [F,3,H,W] -> [F, H/patch, W/patch]."""
+    img = np.asarray(images, dtype=np.float64)
+    f, c, h, w = img.shape
+    assert c == 3 and h % patch_px == 0 and w % patch_px == 0
+    grey = (img[:, 0] + img[:, 1] + img[:, 2]) / 3.0
+    pad = np.pad(grey, ((0, 0), (1, 1), (1, 1)), mode="edge")
+    # neighbours of pixel (y,x): pad[y+dy+1, x+dx+1]
+    def nb(dy, dx):
+        return pad[:, 1 + dy:1 + dy + h, 1 + dx:1 + dx + w]
+    gx = (nb(-1, 1) - nb(-1, -1)) + 2.0 * (nb(0, 1) - nb(0, -1)) + (nb(1, 1) - nb(1, -1))
+    gy = (nb(1, -1) - nb(-1, -1)) + 2.0 * (nb(1, 0) - nb(-1, 0)) + (nb(1, 1) - nb(-1, 1))
+    mag = np.sqrt(gx * gx + gy * gy)
+    gh, gw = h // patch_px, w // patch_px
+    return mag.reshape(f, gh, patch_px, gw, patch_px).mean(axis=(2, 4))
+
+
+def var_map(x, frames, grid_h, grid_w, n_special=5, window=3):
+    """Var map Psi_v (Sec. 3.4, "Token Variance"): tokens rearranged to the 2-D patch
+    grid, local average-pooled variance.
+
+    Reading: for every grid position the window is the window x window neighbourhood
+    clipped to the grid; per channel the population variance of the window's values;
+    Psi_v is the mean of that variance over the D channels.  x [N,D] -> [F,gh,gw]."""
+    x = np.asarray(x, dtype=np.float64)
+    t = grid_h * grid_w + n_special
+    d = x.shape[1]
+    grid = x.reshape(frames, t, d)[:, n_special:, :].reshape(frames, grid_h, grid_w, d)
+    half = window // 2
+    out = np.zeros((frames, grid_h, grid_w))
+    for py in range(grid_h):
+        y0, y1 = max(0, py - half), min(grid_h, py + half + 1)
+        for px in range(grid_w):
+            x0, x1 = max(0, px - half), min(grid_w, px + half + 1)
+            win = grid[:, y0:y1, x0:x1, :].reshape(frames, -1, d)
+            mu = win.mean(axis=1, keepdims=True)
+            out[:, py, px] = ((win - mu) ** 2).mean(axis=1).mean(axis=1)
+    return out
+
+
+def ga_map(grad, var, alpha=0.5, beta=0.5, eps=1e-6):
+    """Psi_GA = alpha*norm(Psi_g) + beta*norm(Psi_v) (Sec. 3.4, unnumbered equation).
+    Reading of norm(.): per-frame min-max, (v - min) / (max - min + eps)."""
+    def norm(m):
+        m = np.asarray(m, dtype=np.float64)
+        lo = m.min(axis=(1, 2), keepdims=True)
+        hi = m.max(axis=(1, 2), keepdims=True)
+        return (m - lo) / (hi - lo + eps)
+    return alpha * norm(grad) + beta * norm(var)
+
+
+# --------------------------------------------------------------------------------------
+# step 1 (cont.): partition into GA / dst / src
+# --------------------------------------------------------------------------------------
+def partition(ga, n_special=5, ga_keep_frac=0.10, cell_h=2, cell_w=2):
+    """Token classes (Sec. 3.4, "GA Token Partitioning").
+
+    Frame 0: every patch token is an anchor.  Other frames: cells of cell_h x cell_w
+    anchored at the grid origin and clipped at the far edges; in each cell the patch
+    with the lowest GA score becomes the anchor; among the patches that are not
+    anchors, the floor(frac*P) highest GA scores become GA tokens; the rest are src.
+    Special tokens of every frame are protected.  Returns cls [N] uint8."""
+    ga = np.asarray(ga, dtype=np.float64)
+    frames, gh, gw = ga.shape
+    p = gh * gw
+    t = p + n_special
+    n_ga = int(np.floor(ga_keep_frac * p + 1e-9))
+    cls = np.full(frames * t, CLS_PROTECTED, dtype=np.uint8)
+    for f in range(frames):
+        base = f * t + n_special
+        if f == 0:
+            cls[base:base + p] = CLS_DST
+            continue
+        score = ga[f].reshape(p)
+        is_dst = np.zeros(p, dtype=bool)
+        for cy in range(0, gh, cell_h):
+            for cx in range(0, gw, cell_w):
+                best, best_v = -1, np.inf
+                for py in range(cy, min(gh, cy + cell_h)):
+                    for px in range(cx, min(gw, cx + cell_w)):
+                        if score[py * gw + px] < best_v:
+                            best, best_v = py * gw + px, score[py * gw + px]
+                is_dst[best] = True
+        rest = np.flatnonzero(~is_dst)
+        # highest score first, ties towards the lowest index
+        order = rest[np.lexsort((rest, -score[rest]))]
+        k = min(n_ga, rest.size)
+        frame_cls = np.full(p, CLS_SRC, dtype=np.uint8)
+        frame_cls[is_dst] = CLS_DST
+        frame_cls[order[:k]] = CLS_GA
+        cls[base:base + p] = frame_cls
+    return cls
+
+
+# --------------------------------------------------------------------------------------
+# step 2: src -> dst matching
+# --------------------------------------------------------------------------------------
+def match(x, src_idx, dst_idx, rows=None, norm_eps=1e-12, chunk=2048):
+    """Cosine matching (Sec. 3.4, "Cached Token Merging": src tokens are matched to
+    dst tokens via cosine similarity, each to its most similar dst).
+
+    Candidates are all anchors of all frames.  rows (optional) selects positions in
+    src_idx to evaluate.  Returns (best_dst token index, best_sim, second_sim)."""
+    x = np.asarray(x, dtype=np.float64)
+    src_idx = np.asarray(src_idx, dtype=np.int64)
+    dst_idx = np.asarray(dst_idx, dtype=np.int64)
+    if rows is not None:
+        src_idx = src_idx[np.asarray(rows, dtype=np.int64)]
+    b = x[dst_idx]
+    nb = np.maximum(np.sqrt((b * b).sum(axis=1)), norm_eps)
+    best = np.empty(src_idx.size, dtype=np.int64)
+    sim1 = np.empty(src_idx.size)
+    sim2 = np.full(src_idx.size, -np.inf)
+    for c0 in range(0, src_idx.size, chunk):
+        a = x[src_idx[c0:c0 + chunk]]
+        na = np.maximum(np.sqrt((a * a).sum(axis=1)), norm_eps)
+        sim = (a @ b.T) / (na[:, None] * nb[None, :])
+        j = sim.argmax(axis=1)  # first maximum = lowest anchor index
+        rowsel = np.arange(a.shape[0])
+        sim1[c0:c0 + chunk] = sim[rowsel, j]
+        best[c0:c0 + chunk] = dst_idx[j]
+        if dst_idx.size > 1:
+            sim[rowsel, j] = -np.inf
+            sim2[c0:c0 + chunk] = sim.max(axis=1)
+    return best, sim1, sim2
+
+
+# --------------------------------------------------------------------------------------
+# step 2 (cont.): which src are merged, and the index arrays
+# --------------------------------------------------------------------------------------
+def select_and_index(cls, best_dst, best_sim, n_remove):
+    """Merge indices.
+
+    best_dst / best_sim are given per src token in ascending token order.  The
+    n_remove src tokens with the highest best_sim (ties: lowest token index) are merged
+    into their anchors; n_remove = |Src| is the paper's rule (every src is merged,
+    Sec. 3.4 "Src Tokens").  Kept tokens keep their original order.  Returns
+    dst_of [N] (row of the merged sequence each token maps to), size [M]
+    (1 + number of src merged into the row), kept_idx [M] (token index of each row)."""
+    cls = np.asarray(cls)
+    n = cls.size
+    src_idx = np.flatnonzero(cls == CLS_SRC)
+    best_dst = np.asarray(best_dst, dtype=np.int64)
+    best_sim = np.asarray(best_sim, dtype=np.float64)
+    assert src_idx.size == best_dst.size == best_sim.size
+    assert 0 <= n_remove <= src_idx.size
+    order = np.lexsort((src_idx, -best_sim))  # primary: sim descending; then index
+    merged_pos = np.sort(order[:n_remove])
+    removed = np.zeros(n, dtype=bool)
+    removed[src_idx[merged_pos]] = True
+    kept_idx = np.flatnonzero(~removed)
+    row_of = np.full(n, -1, dtype=np.int64)
+    row_of[kept_idx] = np.arange(kept_idx.size)
+    dst_of = row_of.copy()
+    dst_of[src_idx[merged_pos]] = row_of[best_dst[merged_pos]]
+    assert (dst_of >= 0).all()
+    size = np.bincount(dst_of, minlength=kept_idx.size)
+    return dst_of, size, kept_idx
+
+
+# --------------------------------------------------------------------------------------
+# step 3: merge, step 4 tail: unmerge
+# --------------------------------------------------------------------------------------
+def merge(x, dst_of, n_merged):
+    """x'_d = (x_d + sum_{s in S_d} x_s) / (1 + |S_d|)  (Sec. 3.4, the merge equation).
+    Rows that absorb nothing are returned unchanged."""
+    x = np.asarray(x, dtype=np.float64)
+    dst_of = np.asarray(dst_of, dtype=np.int64)
+    acc = np.zeros((n_merged, x.shape[1]))
+    np.add.at(acc, dst_of, x)
+    size = np.bincount(dst_of, minlength=n_merged).astype(np.float64)
+    return acc / size[:, None]
+
+
+def unmerge(y_merged, dst_of, residual=None):
+    """Token unmerging (Sec. 3.4): every member of {x_d} U S_d receives a copy of the
+    merged row, restoring the original length; optional residual add."""
+    out = np.asarray(y_merged, dtype=np.float64)[np.asarray(dst_of, dtype=np.int64)]
+    if residual is not None:
+        out = out + np.asarray(residual, dtype=np.float64)
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# step 4: global self-attention over the merged sequence
+# --------------------------------------------------------------------------------------
+def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024,
+                     return_parts=False):
+    """Standard multi-head self-attention over the whole (merged) sequence (Sec. 3.1:
+    the frame-global attention concatenates all tokens for full-sequence attention).
+
+    Weights are output-feature-major: qkv = xm @ w_qkv.T + b_qkv with rows [0,D) = Q,
+    [D,2D) = K, [2D,3D) = V; head h owns channels [h*dh,(h+1)*dh).  Per head
+    softmax(Q K^T / sqrt(dh)) V, non-causal, no mask; y = o @ w_o.T + b_o.
+    rows (optional) restricts the queries (all keys/values are still used)."""
+    xm = np.asarray(xm, dtype=np.float64)
+    w_qkv = np.asarray(w_qkv, dtype=np.float64)
+    w_o = np.asarray(w_o, dtype=np.float64)
+    m, d = xm.shape
+    dh = d // heads
+    b_qkv = np.zeros(3 * d) if b_qkv is None else np.asarray(b_qkv, dtype=np.float64)
+    b_o = np.zeros(d) if b_o is None else np.asarray(b_o, dtype=np.float64)
+    qkv = xm @ w_qkv.T + b_qkv
+    q, k, v = qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:]
+    if rows is not None:
+        q = q[np.asarray(rows, dtype=np.int64)]
+    o = np.empty((q.shape[0], d))
+    scale = 1.0 / np.sqrt(dh)
+    for h in range(heads):
+        sl = slice(h * dh, (h + 1) * dh)
+        kh, vh = k[:, sl], v[:, sl]
+        for c0 in range(0, q.shape[0], chunk):
+            s = (q[c0:c0 + chunk, sl] @ kh.T) * scale
+            s -= s.max(axis=1, keepdims=True)
+            p = np.exp(s)
+            p /= p.sum(axis=1, keepdims=True)
+            o[c0:c0 + chunk, sl] = p @ vh
+    y = o @ w_o.T + b_o
+    if return_parts:
+        return y, qkv, o
+    return y
+
+
+# --------------------------------------------------------------------------------------
+# index cache
+# --------------------------------------------------------------------------------------
+def should_refresh(global_layer_idx, recompute_interval=6):
+    """Merge indices are computed once every `recompute_interval` global layers and
+    reused in between (Sec. 3.4: every 6 layers, 4 computations over 24 layers)."""
+    return global_layer_idx % recompute_interval == 0
+
+
+# --------------------------------------------------------------------------------------
+# the whole plan, for convenience in tests and the CPU-baseline timing
+# --------------------------------------------------------------------------------------
+def merge_plan(x, grad, frames, grid_h, grid_w, n_special=5, merge_ratio=0.5,
+               ga_keep_frac=0.10, alpha=0.5, beta=0.5, cell_h=2, cell_w=2, window=3):
+    """Steps 1b-2 end to end.  Returns a dict with every intermediate."""
+    sz = derived_sizes(frames, grid_h, grid_w, n_special, merge_ratio, ga_keep_frac, cell_h, cell_w)
+    var = var_map(x, frames, grid_h, grid_w, n_special, window)
+    ga = ga_map(grad, var, alpha, beta)
+    cls = partition(ga, n_special, ga_keep_frac, cell_h, cell_w)
+    src_idx = np.flatnonzero(cls == CLS_SRC)
+    dst_idx = np.flatnonzero(cls == CLS_DST)
+    assert src_idx.size == sz["n_src"] and dst_idx.size == sz["n_dst"]
+    if src_idx.size:
+        best_dst, sim1, sim2 = match(x, src_idx, dst_idx)
+    else:
+        best_dst = np.zeros(0, dtype=np.int64)
+        sim1 = sim2 = np.zeros(0)
+    dst_of, size, kept_idx = select_and_index(cls, best_dst, sim1, sz["R"])
+    return dict(sizes=sz, var=var, ga=ga, cls=cls, src_idx=src_idx, dst_idx=dst_idx,
+                best_dst=best_dst, best_sim=sim1, second_sim=sim2, dst_of=dst_of, size=size,
+                kept_idx=kept_idx)
