@@ -1,0 +1,188 @@
+/*
+ * litevggt.h - C ABI of the B200 (sm_100a) library for geometry-aware cached token
+ * merging around VGGT's frame-global attention layer (LiteVGGT, Sec. 3.4 of the paper).
+ *
+ * Path (one global layer):
+ *   grad map (once per sequence) -> merge plan [var map + norms -> GA map -> partition
+ *   -> cosine match + row argmax -> select -> index build] -> merge -> global
+ *   attention over the merged tokens -> unmerge.  The plan is the cached index set that
+ *   is reused by the following global layers and refreshed every k-th layer.
+ *
+ * Conventions
+ *   - F frames, patch grid gh x gw, P = gh*gw patch tokens + S special tokens per frame
+ *     (Sec. 3.1: 1 camera + 4 register), T = P + S, N = F*T tokens, D channels.
+ *   - token index i = f*T + t; t < S special, t = S + py*gw + px patch (row-major grid).
+ *   - "dev" pointers are device memory on the ctx's device, "host" pointers are host
+ *     memory.  All tensors are row-major, contiguous and 16-byte aligned
+ *     (LITEVGGT_ERR_ALIGN otherwise).  bf16 tensors are passed as void*.
+ *   - The caller owns every tensor and the stream.  The library owns the ctx workspace
+ *     (allocated once in litevggt_create, sized for the config) and the plan arrays.
+ *   - Every call validates its arguments and returns a status; nothing throws or
+ *     aborts.  Compute calls enqueue work on `stream` (a cudaStream_t passed as void*)
+ *     and return without synchronising, unless stated otherwise.
+ *   - Device-side pipeline waits are bounded; a kernel that gives up records it in the
+ *     ctx's device status word, which litevggt_poll_device_status reads.
+ *   - There is no CPU or non-sm_100 fallback: LITEVGGT_ERR_ARCH on other devices.
+ */
+#ifndef LITEVGGT_H_
+#define LITEVGGT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LITEVGGT_OK = 0,
+  LITEVGGT_ERR_NULL = 1,           /* a required pointer is NULL */
+  LITEVGGT_ERR_BAD_CONFIG = 2,     /* config field out of range / unsupported */
+  LITEVGGT_ERR_SHAPE = 3,          /* a size argument disagrees with the config */
+  LITEVGGT_ERR_ALIGN = 4,          /* a tensor is not 16-byte aligned */
+  LITEVGGT_ERR_ALLOC = 5,          /* device or host allocation failed */
+  LITEVGGT_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed */
+  LITEVGGT_ERR_ARCH = 7,           /* device is not compute capability 10.x */
+  LITEVGGT_ERR_STALE_PLAN = 8,     /* plan belongs to another ctx, or was never built */
+  LITEVGGT_ERR_DEVICE_TIMEOUT = 9, /* a kernel gave up on a bounded wait */
+  LITEVGGT_ERR_DEVICE_BOUNDS = 10  /* a kernel met an out-of-range index and skipped it */
+} litevggt_status;
+
+/* Token classes written by the partition (Sec. 3.4, "GA Token Partitioning"). */
+enum {
+  LITEVGGT_CLS_PROTECTED = 0, /* special tokens: never merged, never anchors */
+  LITEVGGT_CLS_GA = 1,        /* top geometric-importance tokens: excluded from merging */
+  LITEVGGT_CLS_DST = 2,       /* anchors */
+  LITEVGGT_CLS_SRC = 3        /* merge candidates */
+};
+
+typedef struct {
+  int32_t frames;             /* F >= 1 */
+  int32_t grid_h, grid_w;     /* patch grid; image is (14*grid_h) x (14*grid_w) pixels */
+  int32_t patch_px;           /* 14 */
+  int32_t n_special;          /* 5 (1 camera + 4 register tokens, ahead of the patches) */
+  int32_t dim;                /* 1024 */
+  int32_t heads;              /* 16 (head dim must be 64) */
+  float merge_ratio;          /* r in [0,1]: R = min(|Src|, floor(r*N)) src tokens are merged
+                                 away, most similar first.  r >= |Src|/N is the paper's
+                                 rule (every src token is merged); r = 0 is the identity. */
+  float ga_keep_frac;         /* 0.10: fraction of patches per frame kept as GA tokens */
+  float alpha, beta;          /* 0.5, 0.5: weights of norm(Grad map), norm(Var map) */
+  int32_t cell_h, cell_w;     /* 2, 2: one anchor per cell in frames 1..F-1 */
+  int32_t var_window;         /* 3: window of the Var map */
+  int32_t recompute_interval; /* 6: refresh the plan every this many global layers */
+  int32_t qkv_dtype;          /* 0 = bf16 (only value supported) */
+} litevggt_config;
+
+typedef struct litevggt_ctx litevggt_ctx;   /* workspace, tensor maps, device status word */
+typedef struct litevggt_plan litevggt_plan; /* the cached merge indices */
+
+/* Fill `cfg` with the paper's defaults for the given sequence shape. */
+litevggt_status litevggt_default_config(int32_t frames, int32_t grid_h, int32_t grid_w,
+                                        float merge_ratio, litevggt_config* cfg);
+
+/* Create a context on `device`: validates the config, allocates the workspace, builds
+ * the tensor maps.  Synchronous.  *out is NULL on failure. */
+litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt_ctx** out);
+litevggt_status litevggt_destroy(litevggt_ctx* ctx);
+
+/* Sizes that follow from the config (host arithmetic only; any output may be NULL):
+ * N tokens, M merged rows, |Src|, |Dst|, bytes of device workspace held by the ctx. */
+litevggt_status litevggt_sizes(const litevggt_ctx* ctx, int64_t* n_tokens, int64_t* n_merged,
+                               int64_t* n_src, int64_t* n_dst, size_t* workspace_bytes);
+
+/* Grad map (Sec. 3.4, "Pixel Gradient"): Sobel on the channel-mean intensity with
+ * replicate padding, magnitude, mean over each patch.
+ * images: dev fp32 [F,3,14*gh,14*gw] in [0,1];  grad: dev fp32 [F,gh,gw] (written). */
+litevggt_status litevggt_grad_map(litevggt_ctx* ctx, const float* images, float* grad, void* stream);
+
+/* Merge plan (Sec. 3.4): Var map of x (3x3 clipped window, population variance per
+ * channel, mean over channels), GA map = alpha*norm(grad)+beta*norm(var) with per-frame
+ * min-max normalisation, partition into GA/dst/src tokens, cosine matching of every
+ * src token against all anchors of all frames (row argmax, ties to the lowest anchor),
+ * selection of the R most similar src tokens and the index arrays.
+ * x: dev bf16 [N,D] (read);  grad: dev fp32 [F,gh,gw] (read).
+ * *plan_inout == NULL: a plan is created; otherwise it is refreshed in place. */
+litevggt_status litevggt_merge_plan(litevggt_ctx* ctx, const void* x, const float* grad,
+                                    litevggt_plan** plan_inout, void* stream);
+
+/* Same as litevggt_merge_plan from the matching step onwards, with the partition given
+ * by the caller (cls: dev uint8 [N], LITEVGGT_CLS_* values with exactly the per-frame
+ * class counts the config implies; LITEVGGT_ERR_DEVICE_BOUNDS is flagged otherwise).
+ * Used for stage-isolated tests and for other anchor rules. */
+litevggt_status litevggt_merge_plan_with_partition(litevggt_ctx* ctx, const void* x,
+                                                   const uint8_t* cls, litevggt_plan** plan_inout,
+                                                   void* stream);
+
+/* Merge (Sec. 3.4, merge equation): x'_d = (x_d + sum_{s in S_d} x_s) / (1 + |S_d|),
+ * fp32 accumulation in ascending token order, one rounding to bf16; rows that absorb
+ * nothing are copied bit-exactly.  x: dev bf16 [N,D];  x_merged: dev bf16 [M,D]. */
+litevggt_status litevggt_merge(litevggt_ctx* ctx, const litevggt_plan* plan, const void* x,
+                               void* x_merged, void* stream);
+
+/* Global self-attention over the merged sequence (Sec. 3.1): qkv = x' W_qkv^T + b_qkv,
+ * per head softmax(Q K^T / sqrt(64)) V (non-causal), y' = o W_o^T + b_o.
+ * x_merged: dev bf16 [m,D]; m must equal M.  w_qkv: dev bf16 [3D,D], rows [0,D) Q,
+ * [D,2D) K, [2D,3D) V, head h = channels [64h,64h+64);  b_qkv: dev bf16 [3D] or NULL;
+ * w_o: dev bf16 [D,D] (output-feature-major);  b_o: dev bf16 [D] or NULL;
+ * y_merged: dev bf16 [m,D] (written). */
+litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, int64_t m,
+                                     const void* w_qkv, const void* b_qkv, const void* w_o,
+                                     const void* b_o, void* y_merged, void* stream);
+
+/* Unmerge (Sec. 3.4, "Token Unmerging"): out_i = y'[dst_of[i]] (+ residual_i).
+ * y_merged: dev bf16 [M,D];  residual: dev bf16 [N,D] or NULL;  out: dev bf16 [N,D]. */
+litevggt_status litevggt_unmerge(litevggt_ctx* ctx, const litevggt_plan* plan, const void* y_merged,
+                                 const void* residual, void* out, void* stream);
+
+/* One whole cached global layer from host memory: copies x (host bf16 [N,D]) to the
+ * device, runs merge -> global attention -> unmerge with residual x, copies the result
+ * to out (host bf16 [N,D]).  Weights are dev pointers as in litevggt_global_attn.
+ * Copies are asynchronous on `stream` when the host buffers are pinned. */
+litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, const litevggt_plan* plan,
+                                           const void* x_host, const void* w_qkv, const void* b_qkv,
+                                           const void* w_o, const void* b_o, void* out_host,
+                                           void* stream);
+
+/* Plain bf16 linear layer on the tensor cores: out[m,n] = a[m,k] w[n,k]^T + bias[n].
+ * a: dev bf16 [m,k]; w: dev bf16 [n,k]; bias: dev bf16 [n] or NULL; out: dev bf16 [m,n].
+ * k and n must be multiples of 64.  This is the projection step of the attention layer. */
+litevggt_status litevggt_linear(litevggt_ctx* ctx, const void* a, int64_t m, int64_t k,
+                                const void* w, int64_t n, const void* bias, void* out, void* stream);
+
+/* Index cache policy (Sec. 3.4: indices are computed once every `recompute_interval`
+ * global layers): *yes = 1 when the plan must be (re)built at this global layer. */
+litevggt_status litevggt_should_refresh(const litevggt_ctx* ctx, const litevggt_plan* plan,
+                                        int32_t global_layer_idx, int32_t* yes);
+
+/* Copy plan contents to host arrays (synchronises `stream`; any output may be NULL):
+ * dst_of [N] merged row of every token; size [M]; kept_idx [M] token index of each row;
+ * cls [N]; best_dst [|Src|] anchor token index per src (ascending src token order);
+ * best_sim [|Src|] its cosine; var / ga [F*P] Var map and GA map (0 for a plan built
+ * from a caller's partition or imported). */
+litevggt_status litevggt_plan_export(litevggt_ctx* ctx, const litevggt_plan* plan, int32_t* dst_of,
+                                     int32_t* size, int32_t* kept_idx, uint8_t* cls, int32_t* best_dst,
+                                     float* best_sim, float* var, float* ga, void* stream);
+
+/* Build a plan from a host dst_of [N] array (tests; synchronous).  The array must map
+ * kept tokens to consecutive rows 0..M-1 in ascending token order. */
+litevggt_status litevggt_plan_import(litevggt_ctx* ctx, const int32_t* dst_of, litevggt_plan** out);
+litevggt_status litevggt_plan_destroy(litevggt_plan* plan);
+
+/* Pointer to an internal device buffer of the last litevggt_global_attn call (tests):
+ * which = 0: qkv bf16 [M,3D];  which = 1: attention output o bf16 [M,D]. */
+litevggt_status litevggt_debug_buffer(litevggt_ctx* ctx, int which, void** dev_ptr, size_t* bytes);
+
+/* Synchronise `stream` and report whether any kernel flagged a bounded-wait timeout or
+ * an out-of-range index since the last poll (the flag is cleared). */
+litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
+
+/* Number of kernels this library has launched on behalf of ctx since creation. */
+litevggt_status litevggt_launch_count(const litevggt_ctx* ctx, int64_t* launches);
+
+const char* litevggt_status_string(litevggt_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LITEVGGT_H_ */

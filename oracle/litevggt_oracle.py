@@ -249,23 +249,14 @@ def unmerge(y_merged, dst_of, residual=None):
 # --------------------------------------------------------------------------------------
 # step 4: global self-attention over the merged sequence
 # --------------------------------------------------------------------------------------
-def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024,
-                     return_parts=False):
-    """Standard multi-head self-attention over the whole (merged) sequence (Sec. 3.1:
-    the frame-global attention concatenates all tokens for full-sequence attention).
-
-    Weights are output-feature-major: qkv = xm @ w_qkv.T + b_qkv with rows [0,D) = Q,
-    [D,2D) = K, [2D,3D) = V; head h owns channels [h*dh,(h+1)*dh).  Per head
-    softmax(Q K^T / sqrt(dh)) V, non-causal, no mask; y = o @ w_o.T + b_o.
-    rows (optional) restricts the queries (all keys/values are still used)."""
-    xm = np.asarray(xm, dtype=np.float64)
-    w_qkv = np.asarray(w_qkv, dtype=np.float64)
-    w_o = np.asarray(w_o, dtype=np.float64)
-    m, d = xm.shape
+def attention_core(qkv, heads=16, rows=None, chunk=1024):
+    """Per head softmax(Q K^T / sqrt(dh)) V, non-causal, no mask, max-subtracted softmax.
+    qkv [M, 3D] with columns [0,D) = Q, [D,2D) = K, [2D,3D) = V; head h owns channels
+    [h*dh, (h+1)*dh) of each.  rows (optional) restricts the queries (all keys/values are
+    still used).  Returns o [len(rows) or M, D]."""
+    qkv = np.asarray(qkv, dtype=np.float64)
+    d = qkv.shape[1] // 3
     dh = d // heads
-    b_qkv = np.zeros(3 * d) if b_qkv is None else np.asarray(b_qkv, dtype=np.float64)
-    b_o = np.zeros(d) if b_o is None else np.asarray(b_o, dtype=np.float64)
-    qkv = xm @ w_qkv.T + b_qkv
     q, k, v = qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:]
     if rows is not None:
         q = q[np.asarray(rows, dtype=np.int64)]
@@ -280,7 +271,28 @@ def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024
             p = np.exp(s)
             p /= p.sum(axis=1, keepdims=True)
             o[c0:c0 + chunk, sl] = p @ vh
-    y = o @ w_o.T + b_o
+    return o
+
+
+def linear(a, w, b=None):
+    """a @ w.T + b with output-feature-major weights w [n_out, n_in]."""
+    y = np.asarray(a, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T
+    if b is not None:
+        y = y + np.asarray(b, dtype=np.float64)
+    return y
+
+
+def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024,
+                     return_parts=False):
+    """Standard multi-head self-attention over the whole (merged) sequence (Sec. 3.1:
+    the frame-global attention concatenates all tokens for full-sequence attention).
+
+    qkv = xm @ w_qkv.T + b_qkv (rows [0,D) of w_qkv produce Q, [D,2D) K, [2D,3D) V),
+    o = attention_core(qkv), y = o @ w_o.T + b_o.  No positional terms, no mask.
+    rows (optional) restricts the queries."""
+    qkv = linear(xm, w_qkv, b_qkv)
+    o = attention_core(qkv, heads, rows, chunk)
+    y = linear(o, w_o, b_o)
     if return_parts:
         return y, qkv, o
     return y

@@ -1,0 +1,134 @@
+// Host-side runtime objects behind the C ABI: context (workspace, device status word,
+// launch counter), plan (cached merge indices) and the launchers of each kernel group.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/litevggt.h"
+
+namespace lv {
+
+struct Sizes {
+  int frames, grid_h, grid_w, n_special, dim, heads;
+  int patches;        // P
+  int tokens_frame;   // T
+  long long n_tokens; // N
+  int n_dst_frame, n_ga_frame, n_src_frame;
+  long long n_src, n_dst;
+  long long n_remove; // R
+  long long n_merged; // M
+};
+
+inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
+
+// One device allocation carved into named regions.
+struct Workspace {
+  uint8_t* base = nullptr;
+  size_t bytes = 0;
+  // scoring
+  float* var_map = nullptr;     // [F*P]
+  float* ga_score = nullptr;    // [F*P]
+  uint8_t* cls = nullptr;       // [N]
+  int* src_list = nullptr;      // [|Src|] token index, ascending
+  int* dst_list = nullptr;      // [|Dst|] token index, ascending
+  // matching
+  __nv_bfloat16* panel_src = nullptr;  // [|Src|, D] packed rows
+  __nv_bfloat16* panel_dst = nullptr;  // [|Dst|, D]
+  float* inv_norm_src = nullptr;       // [|Src|]
+  float* inv_norm_dst = nullptr;       // [round_up(|Dst|,256)]
+  // index build
+  unsigned long long* sort_keys = nullptr;  // [pow2 >= max(|Src|, R)]
+  int* scan_tmp = nullptr;                  // [N] kept flags / scan output
+  int* scan_blocks = nullptr;               // block sums
+  int* row_of = nullptr;                    // [N]
+  // attention
+  __nv_bfloat16* qkv = nullptr;    // [M, 3D]
+  __nv_bfloat16* attn_o = nullptr; // [M, D]
+  // whole-layer-from-host staging
+  __nv_bfloat16* stage_x = nullptr;   // [N, D]
+  __nv_bfloat16* stage_xm = nullptr;  // [M, D]
+  __nv_bfloat16* stage_ym = nullptr;  // [M, D]
+  __nv_bfloat16* stage_out = nullptr; // [N, D]
+  uint32_t* status = nullptr;         // device status word
+};
+
+}  // namespace lv
+
+struct litevggt_ctx {
+  uint32_t magic;
+  litevggt_config cfg;
+  lv::Sizes sz;
+  int device;
+  int num_sms;
+  lv::Workspace ws;
+  long long launches;
+  void* encode_tiled;  // cuTensorMapEncodeTiled, resolved at run time
+};
+
+struct litevggt_plan {
+  uint32_t magic;
+  const litevggt_ctx* owner;
+  int built;
+  int last_refresh_layer;
+  bool has_maps;       // var/ga/best_* valid (plan built by the library's own scoring)
+  uint8_t* base;       // one device allocation
+  int* dst_of;         // [N]
+  int* size;           // [M]
+  int* kept_idx;       // [M]
+  int* seg_off;        // [M+1]
+  int* seg_src;        // [R]
+  int* best_dst;       // [|Src|] anchor token index
+  float* best_sim;     // [|Src|]
+};
+
+namespace lv {
+
+// bits of the device status word
+constexpr uint32_t kStatusTimeout = 1u;
+constexpr uint32_t kStatusBounds = 2u;
+
+constexpr uint32_t kCtxMagic = 0x4c564358u;
+constexpr uint32_t kPlanMagic = 0x4c56504cu;
+
+// tensor_map.cu
+bool resolve_encode_tiled(void** fn);
+// 2-D bf16 tensor [outer, inner] row-major with row pitch `pitch_elems`; box [box_outer, box_inner],
+// 128-byte swizzle, zero fill outside the tensor.
+bool make_tmap_bf16_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
+                       uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer);
+
+// scoring.cu
+cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches);
+cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var, cudaStream_t s, int* launches);
+cudaError_t launch_partition(const litevggt_ctx* ctx, const float* grad, const float* var, float* ga, uint8_t* cls,
+                             cudaStream_t s, int* launches);
+cudaError_t launch_build_lists(const litevggt_ctx* ctx, const uint8_t* cls, int* src_list, int* dst_list,
+                               cudaStream_t s, int* launches);
+
+// similarity.cu
+cudaError_t launch_match(litevggt_ctx* ctx, const __nv_bfloat16* x, int* best_dst, float* best_sim, cudaStream_t s,
+                         int* launches);
+
+// index_build.cu
+cudaError_t launch_index_build(litevggt_ctx* ctx, litevggt_plan* plan, cudaStream_t s, int* launches);
+size_t sort_capacity(long long n);
+
+// merge_unmerge.cu
+cudaError_t launch_merge(const litevggt_ctx* ctx, const litevggt_plan* plan, const __nv_bfloat16* x,
+                         __nv_bfloat16* xm, cudaStream_t s, int* launches);
+cudaError_t launch_unmerge(const litevggt_ctx* ctx, const litevggt_plan* plan, const __nv_bfloat16* ym,
+                           const __nv_bfloat16* residual, __nv_bfloat16* out, cudaStream_t s, int* launches);
+
+// linear.cu
+cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k, const __nv_bfloat16* w,
+                          long long n, const __nv_bfloat16* bias, __nv_bfloat16* out, cudaStream_t s, int* launches);
+
+// attention.cu
+cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long m, __nv_bfloat16* o,
+                                   cudaStream_t s, int* launches);
+
+}  // namespace lv

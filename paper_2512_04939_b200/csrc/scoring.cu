@@ -1,0 +1,328 @@
+// Geometric-importance scoring and anchor selection (Sec. 3.4, "Geometry-aware Feature
+// Map" and "GA Token Partitioning"): Grad map, Var map, GA map, token classes and the
+// ascending src / anchor token lists.  All of this is bandwidth- or latency-bound work;
+// no tensor cores are involved.
+#include "common.cuh"
+#include "runtime.h"
+
+namespace lv {
+
+// ----------------------------------------------------------------------------------------
+// Grad map.  One CTA per (frame, patch row): stages the 16 grey rows it needs (14 + one
+// halo row above and below, replicate padding) in shared memory, then one warp per patch
+// sums the Sobel magnitudes of its 14 x 14 pixels in a fixed order.
+constexpr int kGradThreads = 256;
+
+__global__ void __launch_bounds__(kGradThreads)
+grad_map_kernel(const float* __restrict__ images, float* __restrict__ grad, int grid_h, int grid_w, int patch) {
+  extern __shared__ float grey[];  // [(patch+2)][w+2]
+  const int f = blockIdx.y;
+  const int py = blockIdx.x;
+  const int h = grid_h * patch, w = grid_w * patch;
+  const int pitch = w + 2;
+  const int rows = patch + 2;
+  const size_t plane = (size_t)h * w;
+  const float* img = images + (size_t)f * 3 * plane;
+  for (int idx = threadIdx.x; idx < rows * w; idx += kGradThreads) {
+    const int r = idx / w, xcol = idx - r * w;
+    int y = py * patch - 1 + r;
+    y = y < 0 ? 0 : (y >= h ? h - 1 : y);
+    const size_t o = (size_t)y * w + xcol;
+    const float v = (img[o] + img[plane + o] + img[2 * plane + o]) / 3.0f;
+    grey[r * pitch + xcol + 1] = v;
+    if (xcol == 0) grey[r * pitch] = v;
+    if (xcol == w - 1) grey[r * pitch + w + 1] = v;
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int npix = patch * patch;
+  for (int px = warp; px < grid_w; px += kGradThreads / 32) {
+    float acc = 0.0f;
+    for (int i = lane; i < npix; i += 32) {
+      const int r = i / patch, c = i - r * patch;
+      const float* p = grey + (r + 1) * pitch + px * patch + c + 1;  // centre pixel
+      const float tl = p[-pitch - 1], tc = p[-pitch], tr = p[-pitch + 1];
+      const float ml = p[-1], mr = p[1];
+      const float bl = p[pitch - 1], bc = p[pitch], br = p[pitch + 1];
+      const float gx = (tr - tl) + 2.0f * (mr - ml) + (br - bl);
+      const float gy = (bl - tl) + 2.0f * (bc - tc) + (br - tr);
+      acc += sqrtf(gx * gx + gy * gy);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) grad[((size_t)f * grid_h + py) * grid_w + px] = acc / (float)npix;
+  }
+}
+
+cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches) {
+  const Sizes& z = ctx->sz;
+  const int patch = ctx->cfg.patch_px;
+  const size_t smem = (size_t)(patch + 2) * (z.grid_w * patch + 2) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(grad_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  grad_map_kernel<<<dim3(z.grid_h, z.frames), kGradThreads, smem, s>>>(images, grad, z.grid_h, z.grid_w, patch);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------------
+// Var map.  One CTA per (frame, grid row); thread t owns channels 4t..4t+3 and slides a
+// (<=3) x (<=3) window along the row, keeping the three window columns in registers.
+// Two-pass variance in fp32 (mean first, then squared deviations).  Per-position partial
+// sums are reduced over the 256 threads in a fixed order, so the map is deterministic.
+constexpr int kVarThreads = 256;
+
+struct Col3 {
+  float v[3][4];
+};
+
+__device__ __forceinline__ void load_col(Col3& c, const __nv_bfloat16* row0, int nr, size_t row_pitch, int px) {
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    if (r < nr) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(row0 + r * row_pitch + (size_t)px * 1024);
+      c.v[r][0] = bf16_lo(raw.x);
+      c.v[r][1] = bf16_hi(raw.x);
+      c.v[r][2] = bf16_lo(raw.y);
+      c.v[r][3] = bf16_hi(raw.y);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kVarThreads)
+var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var, int grid_h, int grid_w, int n_special) {
+  extern __shared__ float partial[];  // [grid_w][256]
+  const int f = blockIdx.y, py = blockIdx.x;
+  const int tokens_frame = grid_h * grid_w + n_special;
+  const int r0 = py > 0 ? py - 1 : 0;
+  const int r1 = py < grid_h - 1 ? py + 1 : grid_h - 1;
+  const int nr = r1 - r0 + 1;
+  const size_t row_pitch = (size_t)grid_w * 1024;
+  const __nv_bfloat16* row0 =
+      x + ((size_t)f * tokens_frame + n_special + (size_t)r0 * grid_w) * 1024 + threadIdx.x * 4;
+  Col3 left, mid, right;
+  load_col(mid, row0, nr, row_pitch, 0);
+  if (grid_w > 1) load_col(right, row0, nr, row_pitch, 1);
+  for (int px = 0; px < grid_w; ++px) {
+    const bool has_l = px > 0, has_r = px < grid_w - 1;
+    const float inv_n = 1.0f / (float)(nr * (1 + (has_l ? 1 : 0) + (has_r ? 1 : 0)));
+    float tot = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float sum = 0.0f;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        if (r < nr) {
+          sum += mid.v[r][c];
+          if (has_l) sum += left.v[r][c];
+          if (has_r) sum += right.v[r][c];
+        }
+      }
+      const float mu = sum * inv_n;
+      float ss = 0.0f;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        if (r < nr) {
+          float d = mid.v[r][c] - mu;
+          ss += d * d;
+          if (has_l) { d = left.v[r][c] - mu; ss += d * d; }
+          if (has_r) { d = right.v[r][c] - mu; ss += d * d; }
+        }
+      }
+      tot += ss * inv_n;
+    }
+    partial[px * kVarThreads + threadIdx.x] = tot;
+    left = mid;
+    mid = right;
+    if (px + 2 < grid_w) load_col(right, row0, nr, row_pitch, px + 2);
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int px = warp; px < grid_w; px += kVarThreads / 32) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kVarThreads / 32; ++i) acc += partial[px * kVarThreads + i * 32 + lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) var[((size_t)f * grid_h + py) * grid_w + px] = acc / 1024.0f;
+  }
+}
+
+cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var, cudaStream_t s, int* launches) {
+  const Sizes& z = ctx->sz;
+  const size_t smem = (size_t)z.grid_w * kVarThreads * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  var_map_kernel<<<dim3(z.grid_h, z.frames), kVarThreads, smem, s>>>(x, var, z.grid_h, z.grid_w, z.n_special);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------------
+// GA map + partition.  One CTA per frame.  Per-frame min-max normalisation of both maps,
+// weighted sum, segmented (per cell) argmin for the anchors, then an exact top-k of the
+// remaining patches by rank counting (rank = number of candidates that beat this one,
+// ties towards the lower index); P <= a few thousand, so all of it lives in shared memory.
+constexpr int kPartThreads = 512;
+
+__device__ __forceinline__ float block_reduce_minmax(float v, bool is_max, float* scratch) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, v, o);
+    v = is_max ? fmaxf(v, other) : fminf(v, other);
+  }
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float r = scratch[0];
+  for (int i = 1; i < kPartThreads / 32; ++i) r = is_max ? fmaxf(r, scratch[i]) : fminf(r, scratch[i]);
+  return r;
+}
+
+__global__ void __launch_bounds__(kPartThreads)
+partition_kernel(const float* __restrict__ grad, const float* __restrict__ var, float* __restrict__ ga,
+                 uint8_t* __restrict__ cls, int grid_h, int grid_w, int n_special, int n_ga, int cell_h, int cell_w,
+                 float alpha, float beta) {
+  extern __shared__ float part_smem[];
+  const int p_count = grid_h * grid_w;
+  float* score = part_smem;                                        // [P]
+  uint8_t* is_dst = reinterpret_cast<uint8_t*>(score + p_count);   // [P]
+  __shared__ float scratch[kPartThreads / 32];
+  const int f = blockIdx.x;
+  const float* g = grad + (size_t)f * p_count;
+  const float* v = var + (size_t)f * p_count;
+  float gmin = INFINITY, gmax = -INFINITY, vmin = INFINITY, vmax = -INFINITY;
+  for (int p = threadIdx.x; p < p_count; p += kPartThreads) {
+    gmin = fminf(gmin, g[p]); gmax = fmaxf(gmax, g[p]);
+    vmin = fminf(vmin, v[p]); vmax = fmaxf(vmax, v[p]);
+  }
+  gmin = block_reduce_minmax(gmin, false, scratch);
+  gmax = block_reduce_minmax(gmax, true, scratch);
+  vmin = block_reduce_minmax(vmin, false, scratch);
+  vmax = block_reduce_minmax(vmax, true, scratch);
+  const float gden = gmax - gmin + 1e-6f, vden = vmax - vmin + 1e-6f;
+  for (int p = threadIdx.x; p < p_count; p += kPartThreads) {
+    const float sc = alpha * ((g[p] - gmin) / gden) + beta * ((v[p] - vmin) / vden);
+    score[p] = sc;
+    is_dst[p] = 0;
+    ga[(size_t)f * p_count + p] = sc;
+  }
+  uint8_t* out = cls + (size_t)f * (p_count + n_special);
+  for (int t = threadIdx.x; t < n_special; t += kPartThreads) out[t] = LITEVGGT_CLS_PROTECTED;
+  out += n_special;
+  if (f == 0) {  // the first frame's patches are all anchors
+    for (int p = threadIdx.x; p < p_count; p += kPartThreads) out[p] = LITEVGGT_CLS_DST;
+    return;
+  }
+  __syncthreads();
+  const int cells_w = (grid_w + cell_w - 1) / cell_w, cells_h = (grid_h + cell_h - 1) / cell_h;
+  for (int c = threadIdx.x; c < cells_w * cells_h; c += kPartThreads) {
+    const int cy = (c / cells_w) * cell_h, cx = (c % cells_w) * cell_w;
+    int best = -1;
+    float best_v = INFINITY;
+    for (int yy = cy; yy < min(grid_h, cy + cell_h); ++yy)
+      for (int xx = cx; xx < min(grid_w, cx + cell_w); ++xx) {
+        const float sv = score[yy * grid_w + xx];
+        if (best < 0 || sv < best_v) { best = yy * grid_w + xx; best_v = sv; }
+      }
+    is_dst[best] = 1;
+  }
+  __syncthreads();
+  for (int p = threadIdx.x; p < p_count; p += kPartThreads) {
+    uint8_t c = LITEVGGT_CLS_DST;
+    if (!is_dst[p]) {
+      const float sp = score[p];
+      int rank = 0;
+      for (int q = 0; q < p_count; ++q) {
+        const float sq = score[q];
+        rank += (!is_dst[q] && (sq > sp || (sq == sp && q < p))) ? 1 : 0;
+      }
+      c = rank < n_ga ? LITEVGGT_CLS_GA : LITEVGGT_CLS_SRC;
+    }
+    out[p] = c;
+  }
+}
+
+cudaError_t launch_partition(const litevggt_ctx* ctx, const float* grad, const float* var, float* ga, uint8_t* cls,
+                             cudaStream_t s, int* launches) {
+  const Sizes& z = ctx->sz;
+  const size_t smem = (size_t)z.patches * (sizeof(float) + 1) + 16;
+  cudaError_t e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  partition_kernel<<<z.frames, kPartThreads, smem, s>>>(grad, var, ga, cls, z.grid_h, z.grid_w, z.n_special,
+                                                        z.n_ga_frame, ctx->cfg.cell_h, ctx->cfg.cell_w,
+                                                        ctx->cfg.alpha, ctx->cfg.beta);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------------
+// Token lists.  One CTA per frame: src / anchor tokens of the frame in ascending token
+// order, written at the offsets the per-frame class counts imply.  A frame whose counts
+// differ from the expected ones (possible only with a caller-supplied partition) is
+// flagged in the status word; writes never leave the frame's slot.
+constexpr int kListThreads = 256;
+
+__global__ void __launch_bounds__(kListThreads)
+build_lists_kernel(const uint8_t* __restrict__ cls, int* __restrict__ src_list, int* __restrict__ dst_list,
+                   int p_count, int n_special, int n_src_frame, int n_dst_frame, uint32_t* status) {
+  __shared__ int warp_src[kListThreads / 32], warp_dst[kListThreads / 32];
+  const int f = blockIdx.x;
+  const int tokens_frame = p_count + n_special;
+  const int token0 = f * tokens_frame;
+  const int exp_src = f == 0 ? 0 : n_src_frame;
+  const int exp_dst = f == 0 ? p_count : n_dst_frame;
+  const long long src_base = f == 0 ? 0 : (long long)(f - 1) * n_src_frame;
+  const long long dst_base = f == 0 ? 0 : (long long)p_count + (long long)(f - 1) * n_dst_frame;
+  const int per = (tokens_frame + kListThreads - 1) / kListThreads;
+  const int t0 = threadIdx.x * per, t1 = min(tokens_frame, t0 + per);
+  int ns = 0, nd = 0;
+  for (int t = t0; t < t1; ++t) {
+    const uint8_t c = cls[token0 + t];
+    ns += c == LITEVGGT_CLS_SRC;
+    nd += c == LITEVGGT_CLS_DST;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int xs = ns, xd = nd;  // inclusive warp scans
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int a = __shfl_up_sync(0xffffffffu, xs, o), b = __shfl_up_sync(0xffffffffu, xd, o);
+    if (lane >= o) { xs += a; xd += b; }
+  }
+  if (lane == 31) { warp_src[warp] = xs; warp_dst[warp] = xd; }
+  __syncthreads();
+  int off_s = xs - ns, off_d = xd - nd, tot_s = 0, tot_d = 0;
+  for (int i = 0; i < kListThreads / 32; ++i) {
+    if (i < warp) { off_s += warp_src[i]; off_d += warp_dst[i]; }
+    tot_s += warp_src[i];
+    tot_d += warp_dst[i];
+  }
+  if (tot_s != exp_src || tot_d != exp_dst) {
+    if (threadIdx.x == 0) atomicOr(status, kStatusBounds);
+  }
+  for (int t = t0; t < t1; ++t) {
+    const uint8_t c = cls[token0 + t];
+    if (c == LITEVGGT_CLS_SRC) {
+      if (off_s < exp_src) src_list[src_base + off_s] = token0 + t;
+      ++off_s;
+    } else if (c == LITEVGGT_CLS_DST) {
+      if (off_d < exp_dst) dst_list[dst_base + off_d] = token0 + t;
+      ++off_d;
+    }
+  }
+  // a short frame (flagged above) still gets valid token indices in its unused slots
+  for (int i = tot_s + (int)threadIdx.x; i < exp_src; i += kListThreads) src_list[src_base + i] = token0;
+  for (int i = tot_d + (int)threadIdx.x; i < exp_dst; i += kListThreads) dst_list[dst_base + i] = token0;
+}
+
+cudaError_t launch_build_lists(const litevggt_ctx* ctx, const uint8_t* cls, int* src_list, int* dst_list,
+                               cudaStream_t s, int* launches) {
+  const Sizes& z = ctx->sz;
+  build_lists_kernel<<<z.frames, kListThreads, 0, s>>>(cls, src_list, dst_list, z.patches, z.n_special,
+                                                       z.n_src_frame, z.n_dst_frame, ctx->ws.status);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace lv

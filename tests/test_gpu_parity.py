@@ -1,0 +1,309 @@
+"""GPU parity: every step of the CUDA path against the CPU oracle on the same seeded
+inputs, through the C ABI.  Integer / index work must be bit-exact given the same
+upstream result; floating point obeys the tolerances written beside each check."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from synthdata import WORKLOADS, Workload, make_attention_weights, make_images, make_tokens
+from helpers import bf16_bound, rel_err, to_f64
+
+pytestmark = pytest.mark.gpu
+
+MID = Workload("MID", 8, 16, 16, 0.3, "polygons", 1, 6, 7000)      # N=2088, M=1462: 12 key tiles, ragged
+ODD = Workload("ODD", 5, 9, 11, 0.45, "polygons", 1, 6, 8000)       # odd grid: clipped cells, tiny tail
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import paper_2512_04939_b200 as pkg
+    return pkg
+
+
+def _ctx(lib, wl, **kw):
+    return lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, **kw)
+
+
+_CACHE = {}
+
+
+def _inputs(wl):
+    if wl.name not in _CACHE:
+        img = make_images(wl)
+        tok = make_tokens(wl, img)
+        _CACHE[wl.name] = (img, tok)
+    return _CACHE[wl.name]
+
+
+_PLANS = {}
+
+
+def _oracle_plan(wl):
+    if wl.name not in _PLANS:
+        img, tok = _inputs(wl)
+        grad = O.grad_map(img.numpy())
+        _PLANS[wl.name] = (grad, O.merge_plan(to_f64(tok), grad, wl.frames, wl.grid_h, wl.grid_w,
+                                               merge_ratio=wl.merge_ratio))
+    return _PLANS[wl.name]
+
+
+# ------------------------------------------------------------------ a1 grad map
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, WORKLOADS["C2"]], ids=lambda w: w.name)
+def test_grad_map(lib, wl):
+    img, _ = _inputs(wl)
+    ctx = _ctx(lib, wl)
+    got = ctx.grad_map(img.cuda())
+    ctx.poll()
+    ref = O.grad_map(img.numpy())
+    # fp32 arithmetic on O(1) values, 196-term means: 1e-5 relative to the map's scale
+    assert np.abs(to_f64(got) - ref).max() <= 1e-5 * max(ref.max(), 1e-3)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ a2/a3 scoring + partition
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
+def test_var_map_and_partition(lib, wl):
+    img, tok = _inputs(wl)
+    grad, ref = _oracle_plan(wl)
+    ctx = _ctx(lib, wl)
+    plan = ctx.merge_plan(tok.cuda(), torch.from_numpy(grad.astype(np.float32)).cuda())
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    # Var map: fp32 two-pass variance vs float64, relative to the map's scale
+    assert np.abs(ex["var"] - ref["var"]).max() <= 2e-5 * ref["var"].max()
+    assert np.abs(ex["ga"] - ref["ga"]).max() <= 1e-5
+    # classes: the per-frame counts are exact; tokens may differ only where the deciding
+    # score gap is below 1e-5 (fp32 vs fp64 scores), and 99.9 % must agree overall
+    cls = ex["cls"]
+    sz = ref["sizes"]
+    per_frame = cls.reshape(wl.frames, -1)
+    assert np.all(per_frame[:, :5] == O.CLS_PROTECTED)
+    assert np.all(per_frame[0, 5:] == O.CLS_DST)
+    for f in range(1, wl.frames):
+        assert (per_frame[f] == O.CLS_DST).sum() == sz["n_dst_frame"]
+        assert (per_frame[f] == O.CLS_GA).sum() == sz["n_ga_frame"]
+        assert (per_frame[f] == O.CLS_SRC).sum() == sz["n_src_frame"]
+    diff = np.flatnonzero(cls != ref["cls"])
+    assert diff.size <= 1e-3 * cls.size
+    if diff.size:
+        ga = ref["ga"].reshape(wl.frames, -1)
+        for i in diff:
+            f, t = divmod(int(i), wl.tokens_per_frame)
+            others = np.delete(ga[f], t - 5)
+            assert np.abs(others - ga[f, t - 5]).min() < 1e-5, "class differs without a near-tie"
+    plan.destroy()
+    ctx.close()
+
+
+# ------------------------------------------------------------------ a4 matching (stage-isolated)
+def _check_match(ex, ref):
+    agree = ex["best_dst"] == ref["best_dst"]
+    margin = ref["best_sim"] - ref["second_sim"]
+    assert np.all(agree[margin > 1e-3]), "argmax differs although the oracle's margin exceeds 1e-3"
+    assert agree.mean() >= 0.999
+    # a differing index must still be a near-tie: its similarity within 1e-5 of the best
+    assert np.abs(ex["best_sim"] - ref["best_sim"]).max() <= 1e-5
+    return agree.mean(), margin
+
+
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
+def test_match_with_oracle_partition(lib, wl):
+    _, tok = _inputs(wl)
+    _, ref = _oracle_plan(wl)
+    ctx = _ctx(lib, wl)
+    plan = ctx.merge_plan_with_partition(tok.cuda(), torch.from_numpy(ref["cls"]).cuda())
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    _check_match(ex, ref)
+    plan.destroy()
+    ctx.close()
+
+
+# ------------------------------------------------------------------ a5 selection + index arrays
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
+def test_index_build_bit_exact_given_same_matches(lib, wl):
+    _, tok = _inputs(wl)
+    _, ref = _oracle_plan(wl)
+    ctx = _ctx(lib, wl)
+    plan = ctx.merge_plan_with_partition(tok.cuda(), torch.from_numpy(ref["cls"]).cuda())
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    dst_of, size, kept = O.select_and_index(ref["cls"], ex["best_dst"], ex["best_sim"], ref["sizes"]["R"])
+    assert np.array_equal(ex["dst_of"], dst_of)
+    assert np.array_equal(ex["size"], size)
+    assert np.array_equal(ex["kept_idx"], kept)
+    # and when the matches agree with the oracle's, so does the whole plan
+    if np.array_equal(ex["best_dst"], ref["best_dst"]) and ref["sizes"]["R"] == ref["sizes"]["n_src"]:
+        assert np.array_equal(ex["dst_of"], ref["dst_of"])
+    plan.destroy()
+    ctx.close()
+
+
+def test_identity_at_ratio_zero_and_reuse_equals_recompute(lib):
+    wl = WORKLOADS["C1"]
+    img, tok = _inputs(wl)
+    grad = torch.from_numpy(O.grad_map(img.numpy()).astype(np.float32)).cuda()
+    x = tok.cuda()
+    ctx0 = lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, 0.0)
+    p0 = ctx0.merge_plan(x, grad)
+    ex = ctx0.plan_export(p0)
+    assert ctx0.n_merged == ctx0.n_tokens and np.array_equal(ex["dst_of"], np.arange(ctx0.n_tokens))
+    assert torch.equal(ctx0.merge(p0, x), x)
+    ctx0.poll()
+    p0.destroy(); ctx0.close()
+    ctx = _ctx(lib, wl)
+    p = ctx.merge_plan(x, grad)
+    a = ctx.plan_export(p)
+    ctx.merge_plan(x, grad, p)  # refresh in place on unchanged features
+    b = ctx.plan_export(p)
+    for k in ("dst_of", "size", "kept_idx", "cls", "best_dst"):
+        assert np.array_equal(a[k], b[k]), k
+    assert [l for l in range(24) if ctx.should_refresh(p, l)] == [0, 6, 12, 18]
+    assert ctx.should_refresh(None, 3)
+    ctx.poll()
+    p.destroy(); ctx.close()
+
+
+# ------------------------------------------------------------------ a6 / a10 merge, unmerge
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
+def test_merge_unmerge_with_oracle_plan(lib, wl):
+    _, tok = _inputs(wl)
+    _, ref = _oracle_plan(wl)
+    ctx = _ctx(lib, wl)
+    plan = ctx.plan_import(ref["dst_of"])
+    x = tok.cuda()
+    xm = ctx.merge(plan, x)
+    ctx.poll()
+    x64 = to_f64(tok)
+    ref_m = O.merge(x64, ref["dst_of"], ref["sizes"]["M"])
+    got = to_f64(xm)
+    assert rel_err(got, ref_m) <= bf16_bound(ref_m)
+    single = ref["size"] == 1
+    assert np.array_equal(got[single], x64[ref["kept_idx"][single]])  # bit-exact copies
+    # conservation of size-weighted sums, up to the one bf16 rounding per merged row
+    lhs = (ref["size"][:, None] * got).sum(0)
+    assert np.abs(lhs - x64.sum(0)).max() <= 2.0 ** -8 * np.abs(x64).sum(0).max()
+    # unmerge: pure gather is bit-exact; with residual one fp32 add + rounding
+    ym = torch.randn(ctx.n_merged, 1024, generator=torch.Generator().manual_seed(5)).to(torch.bfloat16).cuda()
+    out = ctx.unmerge(plan, ym)
+    assert np.array_equal(to_f64(out), O.unmerge(to_f64(ym), ref["dst_of"]))
+    out_r = ctx.unmerge(plan, ym, x)
+    ref_r = O.unmerge(to_f64(ym), ref["dst_of"], x64)
+    assert rel_err(to_f64(out_r), ref_r) <= bf16_bound(ref_r)
+    ctx.poll()
+    plan.destroy()
+    ctx.close()
+
+
+# ------------------------------------------------------------------ a7 / a9 projections
+@pytest.mark.parametrize("m,k,n", [(543, 1024, 3072), (1462, 1024, 1024), (5, 64, 64), (300, 128, 320)])
+def test_linear(lib, m, k, n):
+    wl = WORKLOADS["C1"]
+    ctx = _ctx(lib, wl)
+    g = torch.Generator().manual_seed(m + n)
+    a = torch.randn(m, k, generator=g).to(torch.bfloat16)
+    w = (0.05 * torch.randn(n, k, generator=g)).to(torch.bfloat16)
+    b = (0.1 * torch.randn(n, generator=g)).to(torch.bfloat16)
+    for bias in (b, None):
+        got = ctx.linear(a.cuda(), w.cuda(), None if bias is None else bias.cuda())
+        ctx.poll()
+        ref = to_f64(a) @ to_f64(w).T + (0 if bias is None else to_f64(bias))
+        assert rel_err(to_f64(got), ref) <= bf16_bound(ref)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ a7-a9 attention
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
+def test_global_attention(lib, wl):
+    _, tok = _inputs(wl)
+    _, ref = _oracle_plan(wl)
+    m = ref["sizes"]["M"]
+    xm = torch.from_numpy(O.merge(to_f64(tok), ref["dst_of"], m).astype(np.float32)).to(torch.bfloat16)
+    w_qkv, b_qkv, w_o, b_o = make_attention_weights(wl, 0)
+    # second pass with 3x larger projection weights: the softmax becomes far from uniform
+    # (random-init 0.02 weights alone give nearly flat attention, which would hide
+    # indexing mistakes)
+    w_big = (w_qkv.float() * 3.0).to(torch.bfloat16)
+    ctx = _ctx(lib, wl)
+    for wq in (w_qkv, w_big):
+        y = ctx.global_attn(xm.cuda(), wq.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
+        ctx.poll()
+        # each stage against the oracle fed with the GPU's own upstream (bf16) result
+        ref_qkv = O.linear(to_f64(xm), to_f64(wq), to_f64(b_qkv))
+        qkv = to_f64(ctx.debug_buffer(0))
+        assert rel_err(qkv, ref_qkv) <= bf16_bound(ref_qkv), "qkv projection"
+        ref_o = O.attention_core(qkv, heads=16)
+        o = to_f64(ctx.debug_buffer(1))
+        assert rel_err(o, ref_o) <= bf16_bound(ref_o), "attention core"
+        ref_y = O.linear(o, to_f64(w_o), to_f64(b_o))
+        assert rel_err(to_f64(y), ref_y) <= bf16_bound(ref_y), "output projection"
+        if wq is w_qkv:  # end to end (bf16 intermediates on the GPU side, none in the oracle)
+            ref_full = O.global_attention(to_f64(xm), to_f64(wq), to_f64(b_qkv), to_f64(w_o), to_f64(b_o), heads=16)
+            assert rel_err(to_f64(y), ref_full) <= bf16_bound(ref_full), "attention layer end to end"
+    ctx.close()
+
+
+# ------------------------------------------------------------------ whole layer
+def test_whole_layer_c1_and_host_entry(lib):
+    wl = WORKLOADS["C1"]
+    img, tok = _inputs(wl)
+    ctx = _ctx(lib, wl)
+    x = tok.cuda()
+    grad = ctx.grad_map(img.cuda())
+    plan = ctx.merge_plan(x, grad)
+    w = [t.cuda() for t in make_attention_weights(wl, 0)]
+    xm = ctx.merge(plan, x)
+    ym = ctx.global_attn(xm, *w)
+    out = ctx.unmerge(plan, ym, x)
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    x64 = to_f64(tok)
+    ref_m = O.merge(x64, ex["dst_of"], ctx.n_merged)
+    ref_y = O.global_attention(ref_m, *[to_f64(t) for t in w], heads=16)
+    ref_out = O.unmerge(ref_y, ex["dst_of"], x64)
+    assert rel_err(to_f64(out), ref_out) <= bf16_bound(ref_out)
+    x_host = tok.clone().pin_memory()
+    out_host = torch.empty_like(x_host).pin_memory()
+    ctx.global_layer_host(plan, x_host, *w, out_host)
+    ctx.poll()
+    assert torch.equal(out_host, out.cpu())
+    assert ctx.launch_count() > 10
+    plan.destroy()
+    ctx.close()
+
+
+# ------------------------------------------------------------------ ABI misuse
+def test_abi_misuse_returns_error_codes(lib):
+    wl = WORKLOADS["C1"]
+    _, tok = _inputs(wl)
+    ctx = _ctx(lib, wl)
+    other = lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, 0.25)
+    x = tok.cuda()
+    _, ref = _oracle_plan(wl)
+    plan = ctx.plan_import(ref["dst_of"])
+    with pytest.raises(lib.LiteVGGTError) as e:
+        other.merge(plan, x, torch.empty(other.n_merged, 1024, dtype=torch.bfloat16, device="cuda"))
+    assert e.value.code == 8  # stale / foreign plan
+    with pytest.raises(lib.LiteVGGTError) as e:
+        lib.binding._check(ctx.lib.litevggt_global_attn(ctx.handle, x.data_ptr(), 17, x.data_ptr(), None,
+                                                        x.data_ptr(), None, x.data_ptr(), None), "global_attn")
+    assert e.value.code == 3  # shape
+    with pytest.raises(lib.LiteVGGTError) as e:
+        lib.binding._check(ctx.lib.litevggt_merge(ctx.handle, plan.handle, x.data_ptr() + 2, x.data_ptr(), None), "merge")
+    assert e.value.code == 4  # alignment
+    bad = ref["dst_of"].copy()
+    bad[0] = ctx.n_merged + 5
+    with pytest.raises(lib.LiteVGGTError) as e:
+        ctx.plan_import(bad)
+    assert e.value.code == 3
+    # a caller partition with wrong class counts is flagged, not followed out of bounds
+    cls_bad = torch.from_numpy(ref["cls"].copy())
+    cls_bad[wl.tokens_per_frame + 7] = O.CLS_PROTECTED if cls_bad[wl.tokens_per_frame + 7] != O.CLS_PROTECTED else O.CLS_SRC
+    p2 = ctx.merge_plan_with_partition(x, cls_bad.cuda())
+    with pytest.raises(lib.LiteVGGTError) as e:
+        ctx.poll()
+    assert e.value.code == 10
+    ctx.poll()  # flag was cleared
+    p2.destroy(); plan.destroy()
+    other.close(); ctx.close()
