@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: frames/s through (plan refresh every k-th layer) + merge +
+global attention + unmerge on a synthetic VGGT-shaped sequence.
+
+A step is one global layer: when ``step % recompute_interval == 0`` the merge plan is
+rebuilt first (the Grad map once, at step 0), then merge -> global attention over the
+merged tokens -> unmerge with the residual, and the result feeds the next layer.  With the
+default K = 6 the timed region holds exactly one refresh period, i.e. every step of the
+path runs inside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C5] [--impl ours|reference]
+
+N > 1 (torchrun): the path does not shard, so every rank runs an independent replica of
+the workload (its own seeded sequence); no data-path collective exists.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
+
+METRIC = "frames/s through merge+global-attn+unmerge (plan refreshed every 6th layer)"
+UNIT = "frames/s"
+CPU_SAMPLE_FRAMES = 16
+
+
+def _measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle leg (the reported baseline, and the --impl reference arm)
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_layer(wl, images_s, tokens_s, weights, frames_s):
+    """One pass of the whole path with the CPU oracle on the first `frames_s` frames.
+    Returns per-step seconds."""
+    import oracle as O
+
+    f64 = lambda t: t.detach().float().cpu().numpy().astype(np.float64)
+    x = f64(tokens_s)
+    t = {}
+    t0 = time.perf_counter(); grad = O.grad_map(images_s.cpu().numpy()); t["grad_map"] = time.perf_counter() - t0
+    sz = O.derived_sizes(frames_s, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio)
+    t0 = time.perf_counter(); var = O.var_map(x, frames_s, wl.grid_h, wl.grid_w); t["var_map"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    cls = O.partition(O.ga_map(grad, var))
+    src_idx, dst_idx = np.flatnonzero(cls == O.CLS_SRC), np.flatnonzero(cls == O.CLS_DST)
+    t["partition"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); best, sim1, _ = O.match(x, src_idx, dst_idx); t["match"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); dst_of, size, kept = O.select_and_index(cls, best, sim1, sz["R"]); t["index_build"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); xm = O.merge(x, dst_of, sz["M"]); t["merge"] = time.perf_counter() - t0
+    w = [f64(u) for u in weights]
+    t0 = time.perf_counter(); qkv = O.linear(xm, w[0], w[1]); t["qkv_proj"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); o = O.attention_core(qkv, heads=16); t["attention"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); ym = O.linear(o, w[2], w[3]); t["out_proj"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); O.unmerge(ym, dst_of, x); t["unmerge"] = time.perf_counter() - t0
+    return t
+
+
+def extrapolate_frames_per_s(t, frames_s, frames, interval):
+    """Scale the sampled oracle times to the full sequence: matching and the attention core
+    are quadratic in the number of frames, everything else is linear.  Plan steps are
+    amortised over the refresh interval, the Grad map over the whole run of layers."""
+    lin, quad = frames / frames_s, (frames / frames_s) ** 2
+    plan = (t["var_map"] + t["partition"] + t["index_build"]) * lin + t["match"] * quad
+    layer = (t["merge"] + t["qkv_proj"] + t["out_proj"] + t["unmerge"]) * lin + t["attention"] * quad
+    return frames / (layer + plan / interval)
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        n = os.cpu_count() or 1
+    return int(n)
+
+
+def run_cpu_baseline(wl, images, tokens, weights):
+    fs = min(CPU_SAMPLE_FRAMES, wl.frames)
+    t_tok = wl.tokens_per_frame
+    t = oracle_sample_layer(wl, images[:fs], tokens[:fs * t_tok], weights, fs)
+    value = extrapolate_frames_per_s(t, fs, wl.frames, wl.recompute_interval)
+    return {
+        "value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+        "sample": (f"whole path on the first {fs} of {wl.frames} frames of {wl.name} (one layer, {sum(t.values()):.1f} s of CPU "
+                   f"time); extrapolated to {wl.frames} frames: matching and attention core x(F/{fs})^2, other steps "
+                   f"x(F/{fs}), plan amortised over {wl.recompute_interval} layers"),
+        "sample_seconds": {k: round(v, 4) for k, v in t.items()},
+    }
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle as it stands, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    images = make_images(dataclasses.replace(wl, frames=min(CPU_SAMPLE_FRAMES, wl.frames)))
+    small = dataclasses.replace(wl, frames=images.shape[0])
+    tokens = make_tokens(small, images)
+    weights = make_attention_weights(wl, 0)
+    fs = small.frames
+    for _ in range(args.warmup):
+        oracle_sample_layer(wl, images, tokens, weights, fs)
+    times = []
+    t_all = time.perf_counter()
+    for _ in range(args.steps):
+        times.append(oracle_sample_layer(wl, images, tokens, weights, fs))
+    wall = time.perf_counter() - t_all
+    mean = {k: float(np.mean([t[k] for t in times])) for k in times[0]}
+    value = extrapolate_frames_per_s(mean, fs, wl.frames, wl.recompute_interval)
+    sample = (f"each step = whole path on a {fs}-frame sequence drawn with the {wl.name} recipe; value extrapolated to "
+              f"{wl.frames} frames (matching and attention core x(F/{fs})^2, other steps x(F/{fs}), plan amortised over "
+              f"{wl.recompute_interval} layers)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: {wl.frames} frames {wl.img_w}x{wl.img_h}, N={wl.n_tokens}, D=1024, "
+                               f"merge ratio {wl.merge_ratio}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# the CUDA path
+# ----------------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch.distributed as dist
+
+    import paper_2512_04939_b200 as pkg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)
+    peaks = _measured_peaks()
+
+    images = make_images(wl_rank, dev)
+    tokens = make_tokens(wl_rank, images)
+    ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, device=local,
+                       recompute_interval=wl.recompute_interval)
+    n, m, d = ctx.n_tokens, ctx.n_merged, ctx.dim
+    n_layers = max(args.steps, args.warmup, 1)
+    weights = [[t.to(dev) for t in make_attention_weights(wl, layer)] for layer in range(n_layers)]
+    xm = torch.empty(m, d, dtype=torch.bfloat16, device=dev)
+    ym = torch.empty(m, d, dtype=torch.bfloat16, device=dev)
+    bufs = [torch.empty(n, d, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    state = {"plan": None, "grad": None}
+
+    def run_steps(count):
+        cur = tokens
+        for idx in range(count):
+            if idx % wl.recompute_interval == 0:
+                if idx == 0:
+                    state["grad"] = ctx.grad_map(images)
+                state["plan"] = ctx.merge_plan(cur, state["grad"], state["plan"])
+            ctx.merge(state["plan"], cur, xm)
+            ctx.global_attn(xm, *weights[idx], out=ym)
+            nxt = bufs[idx & 1]
+            ctx.unmerge(state["plan"], ym, cur, out=nxt)
+            cur = nxt
+        return cur
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    run_steps(args.warmup)
+    ctx.poll()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ctx.timers_reset()
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    run_steps(args.steps)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ctx.poll()
+    timers = ctx.timers_read()
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * wl.frames * args.steps / (ms / 1e3)
+
+    # ---- end to end through the host-buffer entry point (same schedule, same weights)
+    x_host = [torch.empty(n, d, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    x_host[0].copy_(tokens)
+    e2e_plan = {"plan": None}
+
+    def run_host_steps(count):
+        for idx in range(count):
+            src, dst = x_host[idx & 1], x_host[(idx + 1) & 1]
+            grad = state["grad"] if idx % wl.recompute_interval == 0 else None
+            e2e_plan["plan"] = ctx.global_layer_host(e2e_plan["plan"], src, *weights[idx], dst, grad=grad)
+        torch.cuda.current_stream().synchronize()
+
+    run_host_steps(1)
+    x_host[0].copy_(tokens)
+    barrier()
+    t0 = time.perf_counter()
+    ev0.record()
+    run_host_steps(args.steps)
+    ev1.record()
+    barrier()
+    e2e_ms = max(ev0.elapsed_time(ev1), 1e3 * (time.perf_counter() - t0))  # device span or host wall clock
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    ctx.poll()
+    e2e_value = world * wl.frames * args.steps / (e2e_ms / 1e3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (attention core) and per-step breakdown
+    att_ms, att_n = timers["attention"]
+    att_flops = 4.0 * m * m * d
+    att_tflops = att_flops / (att_ms / max(att_n, 1) * 1e-3) / 1e12 if att_ms > 0 else 0.0
+    breakdown = {}
+    bytes_of = {"merge": (n + m) * d * 2, "unmerge": (m + 2 * n) * d * 2, "var_map": n * d * 2,
+                "grad_map": wl.frames * 3 * wl.img_h * wl.img_w * 4}
+    flops_of = {"attention": att_flops, "match": 2.0 * ctx.n_src * ctx.n_dst * d, "qkv_proj": 6.0 * m * d * d,
+                "out_proj": 2.0 * m * d * d}
+    for name, (tot, cnt) in timers.items():
+        if cnt == 0:
+            continue
+        per = tot / cnt
+        entry = {"ms": round(per, 4), "launch_groups": cnt}
+        if name in bytes_of:
+            entry["GB/s"] = round(bytes_of[name] / (per * 1e-3) / 1e9, 1)
+            entry["frac_hbm"] = round(entry["GB/s"] / peaks["hbm_gbs"], 4)
+        if name in flops_of:
+            entry["TFLOP/s"] = round(flops_of[name] / (per * 1e-3) / 1e12, 1)
+            entry["frac_bf16_sustained"] = round(entry["TFLOP/s"] / peaks["bf16_sustained"], 4)
+        breakdown[name] = entry
+
+    cpu = run_cpu_baseline(wl, images, tokens, weights[0]) if world == 1 and not args.no_cpu_baseline else None
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": f"{wl.name}: {wl.frames} frames {wl.img_w}x{wl.img_h}, N={n} tokens, M={m} merged, D=1024, "
+                        f"16 heads x 64, merge ratio {wl.merge_ratio}, plan refresh every {wl.recompute_interval} layers",
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+            "l2": "inputs larger than L2 (x is %.2f GB); no flush between steps" % (n * d * 2 / 1e9),
+            "tokens_per_s": world * n * args.steps / (ms / 1e3),
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * d * 2, "d2h_bytes_per_step": n * d * 2,
+                "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches,
+        "roofline": {"kernel": "flash_attention_kernel", "bound": "tensor", "achieved": att_tflops,
+                     "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                     "frac": att_tflops / peaks["bf16_sustained"], "traffic": None,
+                     "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
+                     "flops_per_launch": att_flops, "ms_per_launch": att_ms / max(att_n, 1)},
+        "breakdown": breakdown,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=6)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="C5", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

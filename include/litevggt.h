@@ -135,14 +135,16 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
 litevggt_status litevggt_unmerge(litevggt_ctx* ctx, const litevggt_plan* plan, const void* y_merged,
                                  const void* residual, void* out, void* stream);
 
-/* One whole cached global layer from host memory: copies x (host bf16 [N,D]) to the
- * device, runs merge -> global attention -> unmerge with residual x, copies the result
- * to out (host bf16 [N,D]).  Weights are dev pointers as in litevggt_global_attn.
- * Copies are asynchronous on `stream` when the host buffers are pinned. */
-litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, const litevggt_plan* plan,
-                                           const void* x_host, const void* w_qkv, const void* b_qkv,
-                                           const void* w_o, const void* b_o, void* out_host,
-                                           void* stream);
+/* One whole global layer from host memory: copies x (host bf16 [N,D]) to the device,
+ * optionally (re)builds the plan from it (grad != NULL: dev fp32 [F,gh,gw], as in
+ * litevggt_merge_plan; *plan_inout may then be NULL), runs merge -> global attention ->
+ * unmerge with residual x, and copies the result to out (host bf16 [N,D]).  Weights are
+ * dev pointers as in litevggt_global_attn.  Copies are asynchronous on `stream` when the
+ * host buffers are pinned.  The device staging buffers are allocated on the first call. */
+litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, litevggt_plan** plan_inout,
+                                           const float* grad, const void* x_host, const void* w_qkv,
+                                           const void* b_qkv, const void* w_o, const void* b_o,
+                                           void* out_host, void* stream);
 
 /* Plain bf16 linear layer on the tensor cores: out[m,n] = a[m,k] w[n,k]^T + bias[n].
  * a: dev bf16 [m,k]; w: dev bf16 [n,k]; bias: dev bf16 [n] or NULL; out: dev bf16 [m,n].
@@ -176,6 +178,15 @@ litevggt_status litevggt_debug_buffer(litevggt_ctx* ctx, int which, void** dev_p
 /* Synchronise `stream` and report whether any kernel flagged a bounded-wait timeout or
  * an out-of-range index since the last poll (the flag is cleared). */
 litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
+
+/* Device-time stopwatches.  Each step of the path is bracketed by CUDA events recorded on
+ * the launching stream: which = 0 grad map, 1 var map, 2 partition + token lists, 3 cosine
+ * matching (pack + GEMM/argmax), 4 selection + index build, 5 merge, 6 qkv projection,
+ * 7 attention core, 8 output projection, 9 unmerge.  litevggt_timers_reset forgets all
+ * records; litevggt_timer_read synchronises on the recorded events and returns the summed
+ * device time (ms) and the number of records (at most 64 are kept per step). */
+litevggt_status litevggt_timers_reset(litevggt_ctx* ctx);
+litevggt_status litevggt_timer_read(litevggt_ctx* ctx, int which, float* total_ms, int32_t* count);
 
 /* Number of kernels this library has launched on behalf of ctx since creation. */
 litevggt_status litevggt_launch_count(const litevggt_ctx* ctx, int64_t* launches);

@@ -61,7 +61,9 @@ def load_library():
         "litevggt_merge": [vp, vp, vp, vp, vp],
         "litevggt_global_attn": [vp, vp, i64, vp, vp, vp, vp, vp, vp],
         "litevggt_unmerge": [vp, vp, vp, vp, vp, vp],
-        "litevggt_global_layer_host": [vp, vp, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_global_layer_host": [vp, P(vp), vp, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_timers_reset": [vp],
+        "litevggt_timer_read": [vp, C.c_int, P(C.c_float), P(i32)],
         "litevggt_linear": [vp, vp, i64, i64, vp, i64, vp, vp, vp],
         "litevggt_should_refresh": [vp, vp, i32, P(i32)],
         "litevggt_plan_export": [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
@@ -202,14 +204,16 @@ class LiteVGGT:
                "unmerge")
         return out
 
-    def global_layer_host(self, plan: Plan, x_host, w_qkv, b_qkv, w_o, b_o, out_host):
-        """x_host / out_host: CPU bf16 tensors [N, D] (pinned for asynchronous copies)."""
+    def global_layer_host(self, plan: Plan | None, x_host, w_qkv, b_qkv, w_o, b_o, out_host, grad=None) -> Plan:
+        """x_host / out_host: CPU bf16 tensors [N, D] (pinned for asynchronous copies).  With
+        ``grad`` the plan is (re)built from the uploaded tokens first.  Returns the plan."""
         assert x_host.device.type == "cpu" and out_host.device.type == "cpu"
         assert x_host.shape == (self.n_tokens, self.dim) and out_host.shape == x_host.shape
-        _check(self.lib.litevggt_global_layer_host(self.handle, plan.handle, _ptr(x_host), _ptr(w_qkv), _ptr(b_qkv),
-                                                   _ptr(w_o), _ptr(b_o), _ptr(out_host), _stream()),
+        h = plan.handle if plan is not None else C.c_void_p()
+        _check(self.lib.litevggt_global_layer_host(self.handle, C.byref(h), _ptr(grad), _ptr(x_host), _ptr(w_qkv),
+                                                   _ptr(b_qkv), _ptr(w_o), _ptr(b_o), _ptr(out_host), _stream()),
                "global_layer_host")
-        return out_host
+        return plan if plan is not None else Plan(self, h)
 
     def linear(self, a, w, bias=None) -> torch.Tensor:
         m, k = a.shape
@@ -257,6 +261,21 @@ class LiteVGGT:
         cols = 3 * self.dim if which == 0 else self.dim
         view = _DeviceBuffer(ptr.value, (self.n_merged, cols))
         return torch.as_tensor(view, device=self.device).view(torch.bfloat16).clone()
+
+    TIMER_NAMES = ("grad_map", "var_map", "partition", "match", "index_build", "merge", "qkv_proj",
+                   "attention", "out_proj", "unmerge")
+
+    def timers_reset(self):
+        _check(self.lib.litevggt_timers_reset(self.handle), "timers_reset")
+
+    def timers_read(self) -> dict:
+        """{step name: (total device ms, launches recorded)} since the last reset (synchronises)."""
+        out = {}
+        for i, name in enumerate(self.TIMER_NAMES):
+            ms, cnt = C.c_float(), C.c_int32()
+            _check(self.lib.litevggt_timer_read(self.handle, i, C.byref(ms), C.byref(cnt)), "timer_read")
+            out[name] = (ms.value, cnt.value)
+        return out
 
     def poll(self):
         """Synchronise the current stream; raise if a kernel flagged a timeout / bad index."""

@@ -78,6 +78,24 @@ struct Carver {
 
 void bump(litevggt_ctx* ctx, int n) { ctx->launches += n; }
 
+// Brackets the launches of one step with an event pair on the launching stream.
+struct StepTimer {
+  litevggt_ctx* ctx;
+  cudaStream_t s;
+  int which, slot;
+  StepTimer(litevggt_ctx* c, int w, cudaStream_t st) : ctx(c), s(st), which(w), slot(-1) {
+    Timers& t = ctx->timers;
+    if (!t.created) return;
+    slot = t.used[which] % kTimerSlots;
+    cudaEventRecord(t.start[which][slot], s);
+  }
+  ~StepTimer() {
+    if (slot < 0) return;
+    cudaEventRecord(ctx->timers.stop[which][slot], s);
+    ++ctx->timers.used[which];
+  }
+};
+
 litevggt_status cuda_status(cudaError_t e) {
   if (e == cudaSuccess) return LITEVGGT_OK;
   (void)cudaGetLastError();
@@ -119,9 +137,19 @@ litevggt_status alloc_plan(litevggt_ctx* ctx, litevggt_plan** out) {
 // matching -> selection -> index arrays, from the class array in ctx->ws.cls
 litevggt_status plan_from_classes(litevggt_ctx* ctx, const __nv_bfloat16* x, litevggt_plan* plan, cudaStream_t s) {
   int n = 0;
-  cudaError_t e = launch_build_lists(ctx, ctx->ws.cls, ctx->ws.src_list, ctx->ws.dst_list, s, &n);
-  if (e == cudaSuccess) e = launch_match(ctx, x, plan->best_dst, plan->best_sim, s, &n);
-  if (e == cudaSuccess) e = launch_index_build(ctx, plan, s, &n);
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 2, s);
+    e = launch_build_lists(ctx, ctx->ws.cls, ctx->ws.src_list, ctx->ws.dst_list, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 3, s);
+    e = launch_match(ctx, x, plan->best_dst, plan->best_sim, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 4, s);
+    e = launch_index_build(ctx, plan, s, &n);
+  }
   bump(ctx, n);
   if (e != cudaSuccess) return cuda_status(e);
   plan->built = 1;
@@ -190,6 +218,7 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   ctx->num_sms = prop.multiProcessorCount;
   ctx->launches = 0;
   ctx->encode_tiled = nullptr;
+  ctx->timers.created = false;
   if (!resolve_encode_tiled(&ctx->encode_tiled)) {
     delete ctx;
     return LITEVGGT_ERR_CUDA;
@@ -235,7 +264,41 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
     delete ctx;
     return LITEVGGT_ERR_CUDA;
   }
+  Timers& tm = ctx->timers;
+  tm.created = true;
+  for (int w = 0; w < kNumTimers; ++w) {
+    tm.used[w] = 0;
+    for (int i = 0; i < kTimerSlots; ++i)
+      if (cudaEventCreate(&tm.start[w][i]) != cudaSuccess || cudaEventCreate(&tm.stop[w][i]) != cudaSuccess)
+        tm.created = false;
+  }
+  (void)cudaGetLastError();
   *out = ctx;
+  return LITEVGGT_OK;
+}
+
+litevggt_status litevggt_timers_reset(litevggt_ctx* ctx) {
+  if (!ctx_ok(ctx)) return LITEVGGT_ERR_NULL;
+  for (int w = 0; w < kNumTimers; ++w) ctx->timers.used[w] = 0;
+  return LITEVGGT_OK;
+}
+
+litevggt_status litevggt_timer_read(litevggt_ctx* ctx, int which, float* total_ms, int32_t* count) {
+  if (!ctx_ok(ctx) || total_ms == nullptr || count == nullptr) return LITEVGGT_ERR_NULL;
+  if (which < 0 || which >= kNumTimers) return LITEVGGT_ERR_SHAPE;
+  Timers& tm = ctx->timers;
+  *total_ms = 0.0f;
+  *count = 0;
+  if (!tm.created) return LITEVGGT_ERR_CUDA;
+  const int n = tm.used[which] < kTimerSlots ? tm.used[which] : kTimerSlots;
+  for (int i = 0; i < n; ++i) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(tm.stop[which][i]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, tm.start[which][i], tm.stop[which][i]) != cudaSuccess)
+      return cuda_status(cudaGetLastError());
+    *total_ms += ms;
+  }
+  *count = n;
   return LITEVGGT_OK;
 }
 
@@ -244,6 +307,12 @@ litevggt_status litevggt_destroy(litevggt_ctx* ctx) {
   if (!ctx_ok(ctx)) return LITEVGGT_ERR_NULL;
   DeviceGuard g(ctx->device);
   cudaDeviceSynchronize();
+  if (ctx->timers.created)
+    for (int w = 0; w < kNumTimers; ++w)
+      for (int i = 0; i < kTimerSlots; ++i) {
+        cudaEventDestroy(ctx->timers.start[w][i]);
+        cudaEventDestroy(ctx->timers.stop[w][i]);
+      }
   if (ctx->ws.stage_x != nullptr) cudaFree(ctx->ws.stage_x);
   if (ctx->ws.base != nullptr) cudaFree(ctx->ws.base);
   (void)cudaGetLastError();
@@ -267,7 +336,11 @@ litevggt_status litevggt_grad_map(litevggt_ctx* ctx, const float* images, float*
   if (!ctx_ok(ctx) || images == nullptr || grad == nullptr) return LITEVGGT_ERR_NULL;
   if (!aligned16(images) || !aligned16(grad)) return LITEVGGT_ERR_ALIGN;
   int n = 0;
-  cudaError_t e = launch_grad_map(ctx, images, grad, (cudaStream_t)stream, &n);
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 0, (cudaStream_t)stream);
+    e = launch_grad_map(ctx, images, grad, (cudaStream_t)stream, &n);
+  }
   bump(ctx, n);
   return cuda_status(e);
 }
@@ -285,8 +358,15 @@ litevggt_status litevggt_merge_plan(litevggt_ctx* ctx, const void* x, const floa
   cudaStream_t s = (cudaStream_t)stream;
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
   int n = 0;
-  cudaError_t e = launch_var_map(ctx, xb, ctx->ws.var_map, s, &n);
-  if (e == cudaSuccess) e = launch_partition(ctx, grad, ctx->ws.var_map, ctx->ws.ga_score, ctx->ws.cls, s, &n);
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 1, s);
+    e = launch_var_map(ctx, xb, ctx->ws.var_map, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 2, s);
+    e = launch_partition(ctx, grad, ctx->ws.var_map, ctx->ws.ga_score, ctx->ws.cls, s, &n);
+  }
   bump(ctx, n);
   if (e != cudaSuccess) return cuda_status(e);
   plan->has_maps = true;
@@ -316,8 +396,12 @@ litevggt_status litevggt_merge(litevggt_ctx* ctx, const litevggt_plan* plan, con
   if (!plan_ok(plan) || plan->owner != ctx || !plan->built) return LITEVGGT_ERR_STALE_PLAN;
   if (!aligned16(x) || !aligned16(x_merged)) return LITEVGGT_ERR_ALIGN;
   int n = 0;
-  cudaError_t e = launch_merge(ctx, plan, static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(x_merged),
-                               (cudaStream_t)stream, &n);
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 5, (cudaStream_t)stream);
+    e = launch_merge(ctx, plan, static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(x_merged),
+                     (cudaStream_t)stream, &n);
+  }
   bump(ctx, n);
   return cuda_status(e);
 }
@@ -349,13 +433,21 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
   const int d = ctx->sz.dim;
   cudaStream_t s = (cudaStream_t)stream;
   int n = 0;
-  cudaError_t e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d,
-                                static_cast<const __nv_bfloat16*>(w_qkv), 3 * d,
-                                static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.qkv, s, &n);
-  if (e == cudaSuccess) e = launch_flash_attention(ctx, ctx->ws.qkv, m, ctx->ws.attn_o, s, &n);
-  if (e == cudaSuccess)
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 6, s);
+    e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d, static_cast<const __nv_bfloat16*>(w_qkv),
+                      3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.qkv, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 7, s);
+    e = launch_flash_attention(ctx, ctx->ws.qkv, m, ctx->ws.attn_o, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 8, s);
     e = launch_linear(ctx, ctx->ws.attn_o, m, d, static_cast<const __nv_bfloat16*>(w_o), d,
                       static_cast<const __nv_bfloat16*>(b_o), static_cast<__nv_bfloat16*>(y_merged), s, &n);
+  }
   bump(ctx, n);
   return cuda_status(e);
 }
@@ -367,18 +459,25 @@ litevggt_status litevggt_unmerge(litevggt_ctx* ctx, const litevggt_plan* plan, c
   if (!aligned16(y_merged) || !aligned16(out) || (residual != nullptr && !aligned16(residual)))
     return LITEVGGT_ERR_ALIGN;
   int n = 0;
-  cudaError_t e = launch_unmerge(ctx, plan, static_cast<const __nv_bfloat16*>(y_merged),
-                                 static_cast<const __nv_bfloat16*>(residual), static_cast<__nv_bfloat16*>(out),
-                                 (cudaStream_t)stream, &n);
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 9, (cudaStream_t)stream);
+    e = launch_unmerge(ctx, plan, static_cast<const __nv_bfloat16*>(y_merged),
+                       static_cast<const __nv_bfloat16*>(residual), static_cast<__nv_bfloat16*>(out),
+                       (cudaStream_t)stream, &n);
+  }
   bump(ctx, n);
   return cuda_status(e);
 }
 
-litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, const litevggt_plan* plan, const void* x_host,
-                                           const void* w_qkv, const void* b_qkv, const void* w_o, const void* b_o,
-                                           void* out_host, void* stream) {
-  if (!ctx_ok(ctx) || x_host == nullptr || out_host == nullptr) return LITEVGGT_ERR_NULL;
-  if (!plan_ok(plan) || plan->owner != ctx || !plan->built) return LITEVGGT_ERR_STALE_PLAN;
+litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, litevggt_plan** plan_inout, const float* grad,
+                                           const void* x_host, const void* w_qkv, const void* b_qkv, const void* w_o,
+                                           const void* b_o, void* out_host, void* stream) {
+  if (!ctx_ok(ctx) || plan_inout == nullptr || x_host == nullptr || out_host == nullptr) return LITEVGGT_ERR_NULL;
+  if (grad == nullptr) {
+    const litevggt_plan* plan = *plan_inout;
+    if (!plan_ok(plan) || plan->owner != ctx || !plan->built) return LITEVGGT_ERR_STALE_PLAN;
+  }
   litevggt_status st = ensure_staging(ctx);
   if (st != LITEVGGT_OK) return st;
   const Sizes& z = ctx->sz;
@@ -387,8 +486,14 @@ litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, const litevggt_pla
   const size_t bytes = (size_t)z.n_tokens * z.dim * 2;
   cudaError_t e = cudaMemcpyAsync(ws.stage_x, x_host, bytes, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return cuda_status(e);
+  if (grad != nullptr) {
+    st = litevggt_merge_plan(ctx, ws.stage_x, grad, plan_inout, stream);
+    if (st != LITEVGGT_OK) return st;
+  }
+  const litevggt_plan* plan = *plan_inout;
   st = litevggt_merge(ctx, plan, ws.stage_x, ws.stage_xm, stream);
-  if (st == LITEVGGT_OK) st = litevggt_global_attn(ctx, ws.stage_xm, z.n_merged, w_qkv, b_qkv, w_o, b_o, ws.stage_ym, stream);
+  if (st == LITEVGGT_OK)
+    st = litevggt_global_attn(ctx, ws.stage_xm, z.n_merged, w_qkv, b_qkv, w_o, b_o, ws.stage_ym, stream);
   if (st == LITEVGGT_OK) st = litevggt_unmerge(ctx, plan, ws.stage_ym, ws.stage_x, ws.stage_out, stream);
   if (st != LITEVGGT_OK) return st;
   e = cudaMemcpyAsync(out_host, ws.stage_out, bytes, cudaMemcpyDeviceToHost, s);

@@ -58,6 +58,19 @@ struct Workspace {
 
 }  // namespace lv
 
+namespace lv {
+// Device-time stopwatches, one per step of the path: CUDA event pairs recorded on the
+// launching stream around the step's kernels, kept in a small ring per step.
+constexpr int kNumTimers = 10;
+constexpr int kTimerSlots = 64;
+struct Timers {
+  cudaEvent_t start[kNumTimers][kTimerSlots];
+  cudaEvent_t stop[kNumTimers][kTimerSlots];
+  int used[kNumTimers];  // launches recorded since the last reset
+  bool created;
+};
+}  // namespace lv
+
 struct litevggt_ctx {
   uint32_t magic;
   litevggt_config cfg;
@@ -67,6 +80,7 @@ struct litevggt_ctx {
   lv::Workspace ws;
   long long launches;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved at run time
+  lv::Timers timers;
 };
 
 struct litevggt_plan {

@@ -240,7 +240,9 @@ def test_global_attention(lib, wl):
         assert rel_err(to_f64(y), ref_y) <= bf16_bound(ref_y), "output projection"
         if wq is w_qkv:  # end to end (bf16 intermediates on the GPU side, none in the oracle)
             ref_full = O.global_attention(to_f64(xm), to_f64(wq), to_f64(b_qkv), to_f64(w_o), to_f64(b_o), heads=16)
-            assert rel_err(to_f64(y), ref_full) <= bf16_bound(ref_full), "attention layer end to end"
+            # three stored bf16 intermediates (qkv, o, y) instead of one rounding: the floor of
+            # the chain is about twice that of a single rounding at the 4-5 sigma entries
+            assert rel_err(to_f64(y), ref_full) <= 2 * bf16_bound(ref_full), "attention layer end to end"
     ctx.close()
 
 
@@ -268,6 +270,13 @@ def test_whole_layer_c1_and_host_entry(lib):
     ctx.global_layer_host(plan, x_host, *w, out_host)
     ctx.poll()
     assert torch.equal(out_host, out.cpu())
+    out_host.zero_()
+    plan2 = ctx.global_layer_host(None, x_host, *w, out_host, grad=grad)  # builds its own plan
+    ctx.poll()
+    assert torch.equal(out_host, out.cpu())
+    plan2.destroy()
+    times = ctx.timers_read()
+    assert times["attention"][1] >= 2 and times["attention"][0] > 0.0
     assert ctx.launch_count() > 10
     plan.destroy()
     ctx.close()
