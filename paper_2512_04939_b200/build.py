@@ -18,6 +18,8 @@ CFLAGS = [
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",
     "-I", os.path.join(os.path.dirname(HERE), "include"),
 ]
+# extra nvcc flags (e.g. -DNAME=value to override a tuning constant); changing them needs force=True
+CFLAGS += os.environ.get("LITEVGGT_NVCC_FLAGS", "").split()
 
 
 def _sources():

@@ -42,7 +42,10 @@ constexpr int kFaSmemBytes = (2 + 2 * kFaStages) * kFaTileBytes + 512 + 1024;
 constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColP = 384;
 constexpr float kFaRescaleThreshold = 8.0f;
 // Of every 8 consecutive pairs of scores, this many take the polynomial exponential.
-constexpr int kFaPolyPairsPer8 = 3;
+#ifndef LV_FA_POLY_PAIRS
+#define LV_FA_POLY_PAIRS 2
+#endif
+constexpr int kFaPolyPairsPer8 = LV_FA_POLY_PAIRS;
 
 struct FaBarriers {
   uint64_t q_full;

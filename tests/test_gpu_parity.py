@@ -214,6 +214,20 @@ def test_linear(lib, m, k, n):
 
 
 # ------------------------------------------------------------------ a7-a9 attention
+def attention_core_bound(qkv, ref_o):
+    """Tolerance of the attention core in bf16 arithmetic.  Besides the rounding of the output
+    itself (bf16_bound), the probabilities enter the second tensor-core product as bf16, each
+    with a relative error of up to 2^-9, which moves an output by at most
+    2^-9 * sum_i p_i |v_i| / sum_i p_i.  When a few keys dominate a row the two terms are of
+    the same size, so the second one is part of the bound, evaluated with the oracle on |V|."""
+    d = qkv.shape[1] // 3
+    abs_v = qkv.copy()
+    abs_v[:, 2 * d:] = np.abs(abs_v[:, 2 * d:])
+    weighted_abs = O.attention_core(abs_v, heads=16)
+    rms = float(np.sqrt(np.mean(ref_o * ref_o)))
+    return bf16_bound(ref_o) + 2.0 ** -9 * float(weighted_abs.max()) / rms
+
+
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
 def test_global_attention(lib, wl):
     _, tok = _inputs(wl)
@@ -235,7 +249,7 @@ def test_global_attention(lib, wl):
         assert rel_err(qkv, ref_qkv) <= bf16_bound(ref_qkv), "qkv projection"
         ref_o = O.attention_core(qkv, heads=16)
         o = to_f64(ctx.debug_buffer(1))
-        assert rel_err(o, ref_o) <= bf16_bound(ref_o), "attention core"
+        assert rel_err(o, ref_o) <= attention_core_bound(qkv, ref_o), "attention core"
         ref_y = O.linear(o, to_f64(w_o), to_f64(b_o))
         assert rel_err(to_f64(y), ref_y) <= bf16_bound(ref_y), "output projection"
         if wq is w_qkv:  # end to end (bf16 intermediates on the GPU side, none in the oracle)
