@@ -130,6 +130,30 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
                                      const void* w_qkv, const void* b_qkv, const void* w_o,
                                      const void* b_o, void* y_merged, void* stream);
 
+/* The same attention layer as litevggt_global_attn for callers that must not allocate (the paper
+ * has no counterpart; this is a property of the library, not of the method).  It needs no
+ * context: a context's workspace comes from cudaMalloc, which is off limits for code running
+ * under a memory manager that owns the device, for plug-ins entered after their host froze the
+ * memory map, and for loops that cannot afford the device-wide synchronisation an allocation
+ * brings.  The two intermediates (projected Q/K/V rows and the per-head attention output) live
+ * in a fixed 8 MiB array inside the library image instead, which every GPU that loads the
+ * library holds until the process exits.  Neither this call nor anything it calls allocates or
+ * frees memory.
+ *   - Works on the CURRENT device, for D = 1024 and 16 heads, and for 1 <= m <= 1024 merged rows;
+ *     any other m is refused with LITEVGGT_ERR_SHAPE before anything is launched.
+ *   - The first call on a device looks up the array's device address and the device's
+ *     properties; make that first call outside any stream capture.  Later calls only enqueue.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  The
+ *     call clears what has to start at zero (the status word) itself; two calls whose work
+ *     overlaps on the GPU (different streams, no ordering between them) race on the array.
+ *   - Tensors as in litevggt_global_attn (dev bf16, 16-byte aligned).  device_status: dev pointer
+ *     to one 32-bit word, or NULL; it is zeroed on the stream and afterwards holds 1 if a kernel
+ *     gave up on a bounded wait, 0 otherwise (with NULL the word inside the array is used and
+ *     cannot be read back).  Asynchronous on `stream`. */
+litevggt_status litevggt_global_attn_static(const void* x_merged, int64_t m, const void* w_qkv,
+                                            const void* b_qkv, const void* w_o, const void* b_o,
+                                            void* y_merged, uint32_t* device_status, void* stream);
+
 /* Unmerge (Sec. 3.4, "Token Unmerging"): out_i = y'[dst_of[i]] (+ residual_i).
  * y_merged: dev bf16 [M,D];  residual: dev bf16 [N,D] or NULL;  out: dev bf16 [N,D]. */
 litevggt_status litevggt_unmerge(litevggt_ctx* ctx, const litevggt_plan* plan, const void* y_merged,

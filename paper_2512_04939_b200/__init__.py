@@ -13,6 +13,8 @@ from .binding import (  # noqa: F401
     CLS_GA,
     CLS_DST,
     CLS_SRC,
+    global_attn_static,
+    STATIC_ATTN_MAX_ROWS,
     library_path,
     load_library,
 )

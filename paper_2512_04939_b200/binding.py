@@ -60,6 +60,7 @@ def load_library():
         "litevggt_merge_plan_with_partition": [vp, vp, vp, P(vp), vp],
         "litevggt_merge": [vp, vp, vp, vp, vp],
         "litevggt_global_attn": [vp, vp, i64, vp, vp, vp, vp, vp, vp],
+        "litevggt_global_attn_static": [vp, i64, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_unmerge": [vp, vp, vp, vp, vp, vp],
         "litevggt_global_layer_host": [vp, P(vp), vp, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_timers_reset": [vp],
@@ -97,6 +98,22 @@ def _ptr(t):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+STATIC_ATTN_MAX_ROWS = 1024
+
+
+def global_attn_static(xm, w_qkv, b_qkv, w_o, b_o, out=None, device_status=None):
+    """Attention layer over up to STATIC_ATTN_MAX_ROWS merged rows through the entry point that
+    allocates nothing (no context; intermediates in the library's own fixed device array).  The
+    output tensor is the caller's; pass ``out`` to keep this wrapper from allocating one.
+    ``device_status``: optional int32 CUDA tensor of one element that receives the kernels' flag."""
+    lib = load_library()
+    if out is None:
+        out = torch.empty_like(xm)
+    _check(lib.litevggt_global_attn_static(_ptr(xm), xm.shape[0], _ptr(w_qkv), _ptr(b_qkv), _ptr(w_o), _ptr(b_o),
+                                           _ptr(out), _ptr(device_status), _stream()), "global_attn_static")
+    return out
 
 
 class _DeviceBuffer:
