@@ -4,58 +4,76 @@
 // computed flash-style: scores never leave the SM.
 //
 // One CTA = 256 query rows (two tiles of 128) of one head, sweeping all keys in tiles of
-// 128.  Warp roles (12 warps):
-//   warps 0-3   softmax of query tile 0 (thread = one query row = one TMEM lane)
-//   warps 4-7   softmax of query tile 1
-//   warp  8     MMA issuer (one elected lane):  S_t = Q_t K_j^T  and  O_t += P_t V_j
-//   warp  9     TMA producer (one elected lane): Q once, then K_j / V_j through two
-//               4-stage shared-memory rings
-//   warps 10-11 idle; they only complete the third warpgroup so that the register file can
-//               be re-split (softmax warps take 216 registers, the rest 64)
-// Tensor memory (512 columns): S_0 S_1 (fp32, 128 columns each) | O_0 O_1 (fp32, 64 each)
-// | P_0 P_1 (bf16 pairs, 64 each).  P is fed to the second MMA straight from tensor
-// memory; V tiles are consumed as an MN-major B operand, K tiles as a K-major one, so
-// neither needs a transpose.  While the softmax warps of one tile work, the tensor core
-// runs the other tile's MMAs.
+// 128 that are consumed as two halves of 64 ("steps").  Warp roles (20 warps):
+//   warps 0-15  softmax.  Warp w works on query tile t = w / 8, TMEM lane quarter w % 4 (one
+//               thread = one query row) and the column half c = (w / 4) % 2 of every step:
+//               32 of the step's 64 scores per row.  The two threads of a row swap their
+//               partial row maxima through shared memory once per step.  Four softmax warps
+//               per scheduler keep the special-function unit busy while others wait.
+//   warp  16    MMA issuer of tile 0 (one elected lane):  S_h = Q K_jh^T  and  O += P_h V_jh
+//   warp  17    TMA producer (one elected lane): K_j / V_j through two shared-memory rings
+//   warp  18    MMA issuer of tile 1 (issuing costs tens of cycles per instruction, so one
+//               thread cannot feed both tiles)
+//   warp  19    idle
+// Tensor memory (512 columns allocated, 448 used):
+//   [0,256)    S/P: tile t, half h at column t*128 + h*64.  S_th is 128 x 64 fp32; after the
+//              softmax threads have read it they overwrite its first 32 columns with P_th
+//              (bf16 pairs), which the second MMA reads as its A operand from there.
+//   [256,384)  O_0, O_1 (fp32, 64 columns each)
+//   [384,448)  Q_0, Q_1 (bf16 pairs, 32 columns each), written once by the softmax threads
+//              straight from global memory: Q is the A operand of the first MMA from tensor
+//              memory, so only K and V tiles travel through shared memory.
+// The two halves of a tile double-buffer the scores: while the softmax threads work on
+// half h the tensor core already runs O += P V of the other half and the next Q K^T into
+// it.  The MMAs are issued in order, which is what makes the S/P aliasing safe: Q K^T for
+// step n+2 is issued after the P V that reads the same columns.
+// V tiles are consumed as an MN-major B operand, K tiles as a K-major one, so neither
+// needs a transpose.
 //
 // Softmax arithmetic.  At head dim 64 every score costs 256 tensor flops and one
 // exponential, and the special-function unit issues only 16 ex2 per clock per SM, half of
-// what the tensor cores would need.  So a fixed share of the exponentials of every row is
+// what the tensor cores would need.  A fixed share of the exponentials of every row can be
 // evaluated on the FMA pipes instead: round-to-nearest split x = n + f, |f| <= 1/2, a cubic
 // for 2^f (relative error 7.5e-5, far below the bf16 rounding of P) and n added into the
-// exponent field.  Scale, subtraction of the reference maximum, the polynomial and the row
-// sums use packed two-wide fp32 instructions.
+// exponent field.
 //
 // Online softmax in base 2 with a lazily updated reference maximum: the running output
-// is rescaled only when a row maximum grows by more than 2^8 over the reference, and the
-// final division by the row sum removes the reference again, so the result equals the
-// plain softmax up to rounding.
+// is rescaled only when a row maximum grows by more than 2^8 over the reference (the
+// threads then first wait until the tile's last P V has retired), and the final division
+// by the row sum removes the reference again, so the result equals the plain softmax up
+// to rounding.
 #include "common.cuh"
 #include "runtime.h"
 
 namespace lv {
 
-constexpr int kFaStages = 4;
-constexpr int kFaThreads = 384;
+constexpr int kFaStages = 5;
+constexpr int kFaSoftmaxWarps = 16;
+constexpr int kFaThreads = (kFaSoftmaxWarps + 4) * 32;
 constexpr int kFaTileBytes = 128 * 64 * 2;
-constexpr int kFaSmemBytes = (2 + 2 * kFaStages) * kFaTileBytes + 512 + 1024;
-constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColP = 384;
+constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 384;
 constexpr float kFaRescaleThreshold = 8.0f;
 // Of every 8 consecutive pairs of scores, this many take the polynomial exponential.
 #ifndef LV_FA_POLY_PAIRS
-#define LV_FA_POLY_PAIRS 2
+#define LV_FA_POLY_PAIRS 0
 #endif
 constexpr int kFaPolyPairsPer8 = LV_FA_POLY_PAIRS;
 
 struct FaBarriers {
-  uint64_t q_full;
+  uint64_t q_ready;
   uint64_t k_full[kFaStages], k_empty[kFaStages];
   uint64_t v_full[kFaStages], v_empty[kFaStages];
-  uint64_t s_full[2], p_ready[2], o_done[2];
-  uint64_t teardown;
+  uint64_t s_full[2][2], p_ready[2][2], pv_done[2], o_done[2];
+  uint64_t teardown[2];
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
+// partial row maxima swapped between the two threads of a row: [step parity][tile][column half][row]
+struct FaExchange {
+  float row_max[2][2][2][128];
+  float row_sum[2][2][128];  // [tile][column half][row], once at the end
+};
+constexpr int kFaSmemBytes = 2 * kFaStages * kFaTileBytes + (int)sizeof(FaExchange) + 512 + 1024;
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -98,10 +116,10 @@ __device__ __forceinline__ void drain_ring(uint64_t* full, uint32_t issued, uint
   }
 }
 
-// Exponentials of one 32-score chunk of a row: p = 2^(s * scale - m_ref), packed to bf16
-// pairs; the fp32 values are added to the row's packed partial sums.
+// Exponentials of 32 scores of a row: p = 2^(s * scale - m_ref), packed to bf16 pairs; the fp32
+// values are added to the row's packed partial sums.
 __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 scale2, float2 neg_m2,
-                                              float2 (&sum2)[2], uint32_t (&packed)[16]) {
+                                              float2 (&sum2)[4], uint32_t (&packed)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg_m2);
@@ -112,45 +130,54 @@ __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 sc
       p.x = fast_exp2(x.x);
       p.y = fast_exp2(x.y);
     }
-    sum2[i & 1] = __fadd2_rn(sum2[i & 1], p);
+    sum2[i & 3] = __fadd2_rn(sum2[i & 3], p);
     packed[i] = pack_bf16(p.x, p.y);
   }
 }
 
+__device__ __forceinline__ void pair_barrier(int id) {  // the two warps of one (tile, lane quarter)
+  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+}
+
 __global__ void __launch_bounds__(kFaThreads, 1)
-flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat16* __restrict__ o, int m_rows,
-                       int dim, float scale_log2e, uint32_t* status) {
+flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
+                       __nv_bfloat16* __restrict__ o, int m_rows, int dim, float scale_log2e, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* smem_q = smem;
-  uint8_t* smem_k = smem + 2 * kFaTileBytes;
+  uint8_t* smem_k = smem;
   uint8_t* smem_v = smem_k + kFaStages * kFaTileBytes;
-  FaBarriers* bars = reinterpret_cast<FaBarriers*>(smem_v + kFaStages * kFaTileBytes);
+  FaExchange* xchg = reinterpret_cast<FaExchange*>(smem_v + kFaStages * kFaTileBytes);
+  FaBarriers* bars = reinterpret_cast<FaBarriers*>(xchg + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * 256;
   const int head = blockIdx.y;
   const int n_kv = (m_rows + 127) / 128;
+  const int n_steps = 2 * n_kv;  // step n = key tile n/2, half n%2
 
   if (threadIdx.x == 0) {
-    mbar_init(&bars->q_full, 1);
+    mbar_init(&bars->q_ready, kFaSoftmaxWarps);
     for (int s = 0; s < kFaStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
-      mbar_init(&bars->k_empty[s], 1);
+      mbar_init(&bars->k_empty[s], 2);  // both MMA issuers release a stage
       mbar_init(&bars->v_full[s], 1);
-      mbar_init(&bars->v_empty[s], 1);
+      mbar_init(&bars->v_empty[s], 2);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&bars->s_full[t], 1);
-      mbar_init(&bars->p_ready[t], 4);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(&bars->s_full[t][h], 1);
+        mbar_init(&bars->p_ready[t][h], 8);
+      }
+      mbar_init(&bars->pv_done[t], 1);
       mbar_init(&bars->o_done[t], 1);
     }
-    mbar_init(&bars->teardown, 1);
+    mbar_init(&bars->teardown[0], 1);
+    mbar_init(&bars->teardown[1], 1);
     bars->abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmap_qkv);
   }
-  if (warp == 8) {
+  if (warp == 16) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
   }
@@ -160,187 +187,218 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat
   const uint32_t tmem_base = bars->tmem_base;
   const WaitCtl ctl{&bars->abort_flag, status};
 
-  if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    if (warp == 9) {
-      // ---------------------------------------------------------------- TMA producer
-      if (elect_one()) {
-        mbar_expect_tx(&bars->q_full, 2 * kFaTileBytes);
-        tma_load_2d(smem_q, &tmap_qkv, &bars->q_full, head * 64, q0);
-        tma_load_2d(smem_q + kFaTileBytes, &tmap_qkv, &bars->q_full, head * 64, q0 + 128);
-        uint32_t k_issued = 0, v_issued = 0;
-        for (int j = 0; j < n_kv; ++j) {
-          const int stage = j % kFaStages;
-          const uint32_t phase = (uint32_t)(j / kFaStages) & 1u;
-          if (!mbar_wait(&bars->k_empty[stage], phase ^ 1u, ctl)) break;
-          mbar_expect_tx(&bars->k_full[stage], kFaTileBytes);
-          tma_load_2d(smem_k + stage * kFaTileBytes, &tmap_qkv, &bars->k_full[stage], dim + head * 64, j * 128);
-          ++k_issued;
-          if (!mbar_wait(&bars->v_empty[stage], phase ^ 1u, ctl)) break;
-          mbar_expect_tx(&bars->v_full[stage], kFaTileBytes);
-          tma_load_2d(smem_v + stage * kFaTileBytes, &tmap_qkv, &bars->v_full[stage], 2 * dim + head * 64, j * 128);
-          ++v_issued;
-        }
-        // every load issued by this thread must have landed before the CTA may exit
-        {
-          const long long t0 = clock64();
-          while (!mbar_try_wait(&bars->q_full, 0)) {
-            if (clock64() - t0 > kTimeoutCycles) { atomicOr(status, kStatusTimeout); break; }
-          }
-        }
-        drain_ring(bars->k_full, k_issued, status);
-        drain_ring(bars->v_full, v_issued, status);
+  if (warp == 17) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      uint32_t k_issued = 0, v_issued = 0;
+      for (int j = 0; j < n_kv; ++j) {
+        const int stage = j % kFaStages;
+        const uint32_t phase = (uint32_t)(j / kFaStages) & 1u;
+        if (!mbar_wait(&bars->k_empty[stage], phase ^ 1u, ctl)) break;
+        mbar_expect_tx(&bars->k_full[stage], kFaTileBytes);
+        tma_load_2d(smem_k + stage * kFaTileBytes, &tmap_qkv, &bars->k_full[stage], dim + head * 64, j * 128);
+        ++k_issued;
+        if (!mbar_wait(&bars->v_empty[stage], phase ^ 1u, ctl)) break;
+        mbar_expect_tx(&bars->v_full[stage], kFaTileBytes);
+        tma_load_2d(smem_v + stage * kFaTileBytes, &tmap_qkv, &bars->v_full[stage], 2 * dim + head * 64, j * 128);
+        ++v_issued;
       }
-    } else if (warp == 8) {
-      // ---------------------------------------------------------------- MMA issuer
-      if (elect_one()) {
-        constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
-        constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64, false, true);
-        bool ok = mbar_wait(&bars->q_full, 0, ctl);
-        auto issue_qk = [&](int t, int stage) {
-          const uint64_t a_desc = smem_desc_sw128(smem_u32(smem_q + t * kFaTileBytes), 16, 1024);
-          const uint64_t b_desc = smem_desc_sw128(smem_u32(smem_k + stage * kFaTileBytes), 16, 1024);
+      // every load issued by this thread must have landed before the CTA may exit
+      drain_ring(bars->k_full, k_issued, status);
+      drain_ring(bars->v_full, v_issued, status);
+    }
+  } else if (warp == 16 || warp == 18) {
+    // ------------------------------------------------------------------ MMA issuer of tile t
+    if (elect_one()) {
+      const int t = warp == 16 ? 0 : 1;
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64, false, false);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64, false, true);
+      const uint32_t s_col = tmem_base + kFaColS + t * 128;
+      const uint32_t o_col = tmem_base + kFaColO + t * 64;
+      const uint32_t q_col = tmem_base + kFaColQ + t * 32;
+      // S_h = Q (tensor memory) x K[64h .. 64h+63]^T (shared memory, K-major); 4 steps of 16 channels
+      auto issue_qk = [&](int h, int stage) {
+        const uint64_t b_desc = smem_desc_sw128(smem_u32(smem_k + stage * kFaTileBytes + h * 8192), 16, 1024);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) umma_ts(s_col + h * 64, q_col + k * 8, b_desc + 2 * k, idesc_qk, k != 0 ? 1u : 0u);
+        umma_commit(&bars->s_full[t][h]);
+      };
+      bool ok = mbar_wait(&bars->q_ready, 0, ctl);
+      if (ok) ok = mbar_wait(&bars->k_full[0], 0, ctl);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        issue_qk(1, 0);
+        umma_commit(&bars->k_empty[0]);
+      }
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int j = 0; j < n_kv && ok; ++j) {
+        int next_stage = stage + 1;
+        uint32_t next_phase = phase;
+        if (next_stage == kFaStages) { next_stage = 0; next_phase ^= 1u; }
+        const bool last = j + 1 == n_kv;
+        if (!mbar_wait(&bars->v_full[stage], phase, ctl)) { ok = false; break; }
+        if (!last && !mbar_wait(&bars->k_full[next_stage], next_phase, ctl)) { ok = false; break; }
+        for (int h = 0; h < 2; ++h) {
+          if (!mbar_wait(&bars->p_ready[t][h], j & 1, ctl)) { ok = false; break; }
+          tc_fence_after();
+          // 64 keys of V_j (64 rows of 128 bytes = 8192 bytes per half), 16 keys per instruction:
+          // 8 TMEM columns of P, 2048 bytes of V
+          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192), 1024, 1024);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_ss(tmem_base + kFaColS + t * 128, a_desc + 2 * k, b_desc + 2 * k, idesc_qk, k != 0 ? 1u : 0u);
-          umma_commit(&bars->s_full[t]);
-        };
-        if (ok) ok = mbar_wait(&bars->k_full[0], 0, ctl);
-        if (ok) {
-          tc_fence_after();
-          issue_qk(0, 0);
-          issue_qk(1, 0);
-          umma_commit(&bars->k_empty[0]);
-        }
-        int stage = 0;
-        uint32_t phase = 0;
-        for (int j = 0; j < n_kv && ok; ++j) {
-          int next_stage = stage + 1;
-          uint32_t next_phase = phase;
-          if (next_stage == kFaStages) { next_stage = 0; next_phase ^= 1u; }
-          const bool last = j + 1 == n_kv;
-          if (!mbar_wait(&bars->v_full[stage], phase, ctl)) { ok = false; break; }
-          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes), 1024, 1024);
-          for (int t = 0; t < 2; ++t) {
-            if (!mbar_wait(&bars->p_ready[t], j & 1, ctl)) { ok = false; break; }
-            tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < 8; ++k)  // 16 keys per instruction: 8 TMEM columns of P, 2048 bytes of V
-              umma_ts(tmem_base + kFaColO + t * 64, tmem_base + kFaColP + t * 64 + k * 8, v_desc + 128 * k, idesc_pv,
-                      (j | k) != 0 ? 1u : 0u);
-            if (last) {
-              umma_commit(&bars->o_done[t]);
-            } else {
-              if (t == 0 && !mbar_wait(&bars->k_full[next_stage], next_phase, ctl)) { ok = false; break; }
-              tc_fence_after();
-              issue_qk(t, next_stage);
-              if (t == 1) umma_commit(&bars->k_empty[next_stage]);
-            }
+            umma_ts(o_col, s_col + h * 64 + k * 8, v_desc + 128 * k, idesc_pv, (j | h | k) != 0 ? 1u : 0u);
+          if (last) {
+            // no further Q K^T follows whose completion would tell the softmax threads that this
+            // P V has retired
+            umma_commit(&bars->pv_done[t]);
+            if (h == 1) umma_commit(&bars->o_done[t]);
+          } else {
+            issue_qk(h, next_stage);
           }
-          if (!ok) break;
-          umma_commit(&bars->v_empty[stage]);
-          stage = next_stage;
-          phase = next_phase;
         }
-        if (!ok) {
-          umma_commit(&bars->teardown);
-          const long long t0 = clock64();
-          while (!mbar_try_wait(&bars->teardown, 0)) {
-            if (clock64() - t0 > kTimeoutCycles) break;
-          }
+        if (!ok) break;
+        umma_commit(&bars->v_empty[stage]);
+        if (!last) umma_commit(&bars->k_empty[next_stage]);
+        stage = next_stage;
+        phase = next_phase;
+      }
+      if (!ok) {
+        umma_commit(&bars->teardown[t]);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&bars->teardown[t], 0)) {
+          if (clock64() - t0 > kTimeoutCycles) break;
         }
       }
     }
-  } else {
+  } else if (warp < kFaSoftmaxWarps) {
     // ------------------------------------------------------------------ softmax warps
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-    const int t = warp >> 2;
+    const int t = warp >> 3;
+    const int c = (warp >> 2) & 1;
     const uint32_t quarter = warp & 3u;
+    const int barrier_id = 1 + t * 4 + (int)quarter;
+    const int row_in_tile = (int)quarter * 32 + lane;
     const uint32_t lane_base = (quarter * 32u) << 16;
-    const int row = q0 + t * 128 + (int)quarter * 32 + lane;
+    const int row = q0 + t * 128 + row_in_tile;
     const uint32_t s_addr = tmem_base + lane_base + kFaColS + t * 128;
-    const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * 64;
-    const uint32_t p_addr = tmem_base + lane_base + kFaColP + t * 64;
+    const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * 64 + c * 32;
+    {
+      // this thread's half (32 channels) of its query row goes to tensor memory as it is
+      uint32_t qreg[16];
+      if (row < m_rows) {
+        const uint4* src = reinterpret_cast<const uint4*>(qkv + (size_t)row * 3 * dim + head * 64 + c * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint4 v = __ldg(src + i);
+          qreg[4 * i] = v.x; qreg[4 * i + 1] = v.y; qreg[4 * i + 2] = v.z; qreg[4 * i + 3] = v.w;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) qreg[i] = 0u;
+      }
+      tmem_st16(tmem_base + lane_base + kFaColQ + t * 32 + c * 16, qreg);
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->q_ready);
+    }
     const float2 scale2 = make_float2(scale_log2e, scale_log2e);
     float m_ref = -INFINITY;  // reference maximum, in log2 units (score * scale * log2 e)
-    float2 l_sum2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
+    float2 l_sum2[4] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f),
+                        make_float2(0.0f, 0.0f)};
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      if (!mbar_wait_warp(&bars->s_full[t], j & 1, ctl)) { ok = false; break; }
+    int pair_syncs = 0;  // both warps of a pair must pass the same number of pair barriers
+    for (int n = 0; n < n_steps; ++n) {
+      const int j = n >> 1, h = n & 1;
+      if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
       tc_fence_after();
-      uint32_t s[4][32];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, s[c]);
+      uint32_t s[32];
+      tmem_ld32(s_addr + h * 64 + c * 32, s);
       tmem_ld_wait();
-      const int valid = m_rows - j * 128;
-      if (valid < 128) {
+      const int valid = m_rows - n * 64 - c * 32;
+      if (valid < 32) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i >= valid) s[c][i] = 0xff800000u;  // -inf
+        for (int i = 0; i < 32; ++i)
+          if (i >= valid) s[i] = 0xff800000u;  // -inf
       }
       float mx[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        mx[c] = fmaxf(__uint_as_float(s[c][0]), __uint_as_float(s[c][1]));
-#pragma unroll
-        for (int i = 2; i < 32; i += 2) mx[c] = fmax3(mx[c], __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t* sc = &s[g * 8];
+        mx[g] = fmax3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
+        mx[g] = fmax3(mx[g], __uint_as_float(sc[3]), __uint_as_float(sc[4]));
+        mx[g] = fmax3(mx[g], __uint_as_float(sc[5]), __uint_as_float(sc[6]));
+        mx[g] = fmaxf(mx[g], __uint_as_float(sc[7]));
       }
-      const float mx_scaled = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2e;
-      if (j == 0) {
+      const float mx_own = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
+      // swap with the thread that holds the other 32 scores of this row; this barrier also orders
+      // that thread's P store (into columns this thread has just read) after the read
+      xchg->row_max[n & 1][t][c][row_in_tile] = mx_own;
+      pair_barrier(barrier_id);
+      ++pair_syncs;
+      const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
+      if (n == 0) {
         m_ref = mx_scaled;
       } else {
         const bool grow = mx_scaled > m_ref + kFaRescaleThreshold;
         if (__any_sync(0xffffffffu, grow ? 1 : 0)) {
+          // O_t may still be the target of the previous step's P V.  The issuer follows that P V
+          // with the Q K^T that refills the other half's scores, so their arrival tells that it
+          // has retired; after the last key tile, where nothing follows, pv_done does.
+          const int jp = h == 1 ? j : j - 1;  // key tile of step n-1 (its half is h^1)
+          const bool waited = jp + 1 < n_kv
+                                  ? mbar_wait_warp(&bars->s_full[t][h ^ 1], (uint32_t)(jp + 1) & 1u, ctl)
+                                  : mbar_wait_warp(&bars->pv_done[t], 0, ctl);
+          if (!waited) { ok = false; break; }
+          tc_fence_after();
           const float m_new = grow ? mx_scaled : m_ref;
           const float alpha = fast_exp2(m_ref - m_new);
           const float2 alpha2 = make_float2(alpha, alpha);
-          l_sum2[0] = __fmul2_rn(l_sum2[0], alpha2);
-          l_sum2[1] = __fmul2_rn(l_sum2[1], alpha2);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) l_sum2[i] = __fmul2_rn(l_sum2[i], alpha2);
           m_ref = m_new;
+          uint32_t acc[32];  // this thread's 32 of the row's 64 output channels
+          tmem_ld32(o_addr, acc);
+          tmem_ld_wait();
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            uint32_t acc[32];
-            tmem_ld32(o_addr + c * 32, acc);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * alpha);
-            tmem_st32(o_addr + c * 32, acc);
-          }
+          for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * alpha);
+          tmem_st32(o_addr, acc);
         }
       }
       const float2 neg_m2 = make_float2(-m_ref, -m_ref);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t packed[16];
-        softmax_chunk(s[c], scale2, neg_m2, l_sum2, packed);
-        tmem_st16(p_addr + c * 16, packed);
-      }
+      uint32_t packed[16];
+      softmax_chunk(s, scale2, neg_m2, l_sum2, packed);
+      tmem_st16(s_addr + h * 64 + c * 16, packed);  // P_th lies over the first 32 columns of S_th
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->p_ready[t]);
+      if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
     }
+    // row sums of the two column halves
+    const float l_own = ((l_sum2[0].x + l_sum2[0].y) + (l_sum2[1].x + l_sum2[1].y)) +
+                        ((l_sum2[2].x + l_sum2[2].y) + (l_sum2[3].x + l_sum2[3].y));
+    xchg->row_sum[t][c][row_in_tile] = l_own;
+    // a warp that gave up early still meets its partner at every barrier the partner may be in
+    for (; pair_syncs < n_steps; ++pair_syncs) pair_barrier(barrier_id);
+    pair_barrier(barrier_id);
+    const float l_total = l_own + xchg->row_sum[t][c ^ 1][row_in_tile];
     if (ok && mbar_wait_warp(&bars->o_done[t], 0, ctl)) {
       tc_fence_after();
-      const float inv = 1.0f / ((l_sum2[0].x + l_sum2[0].y) + (l_sum2[1].x + l_sum2[1].y));
+      const float inv = 1.0f / l_total;
+      uint32_t acc[32];
+      tmem_ld32(o_addr, acc);
+      tmem_ld_wait();
+      if (row < m_rows) {
+        uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t acc[32];
-        tmem_ld32(o_addr + c * 32, acc);
-        tmem_ld_wait();
-        if (row < m_rows) {
-          uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(acc[q * 8 + 0]) * inv, __uint_as_float(acc[q * 8 + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(acc[q * 8 + 2]) * inv, __uint_as_float(acc[q * 8 + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(acc[q * 8 + 4]) * inv, __uint_as_float(acc[q * 8 + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(acc[q * 8 + 6]) * inv, __uint_as_float(acc[q * 8 + 7]) * inv);
-            dst[q] = w;
-          }
+        for (int q = 0; q < 4; ++q) {
+          uint4 w;
+          w.x = pack_bf16(__uint_as_float(acc[q * 8 + 0]) * inv, __uint_as_float(acc[q * 8 + 1]) * inv);
+          w.y = pack_bf16(__uint_as_float(acc[q * 8 + 2]) * inv, __uint_as_float(acc[q * 8 + 3]) * inv);
+          w.z = pack_bf16(__uint_as_float(acc[q * 8 + 4]) * inv, __uint_as_float(acc[q * 8 + 5]) * inv);
+          w.w = pack_bf16(__uint_as_float(acc[q * 8 + 6]) * inv, __uint_as_float(acc[q * 8 + 7]) * inv);
+          dst[q] = w;
         }
       }
     }
@@ -348,7 +406,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, __nv_bfloat
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 16) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
@@ -366,7 +424,8 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((m + 255) / 256), (unsigned)ctx->sz.heads);
   const float scale_log2e = 0.125f * 1.4426950408889634f;
-  flash_attention_kernel<<<grid, kFaThreads, kFaSmemBytes, s>>>(tmap, o, (int)m, dim, scale_log2e, ctx->ws.status);
+  flash_attention_kernel<<<grid, kFaThreads, kFaSmemBytes, s>>>(tmap, qkv, o, (int)m, dim, scale_log2e,
+                                                                ctx->ws.status);
   ++*launches;
   return cudaGetLastError();
 }
