@@ -198,6 +198,30 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------------------------
+# rank plumbing (replicas only: no data-path collective, just the timing reduction)
+# ----------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: the job is done when the last replica is."""
+    if world <= 1:
+        return float(ms)
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_frames_per_s(frames: int, steps: int, world: int, ms: float) -> float:
+    """Whole-job throughput: every rank pushes its own `frames`-frame sequence through `steps` layers."""
+    return world * frames * steps / (ms / 1e3)
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each replica draws its own sequence."""
+    return base_seed + 17 * rank
+
+
+# ----------------------------------------------------------------------------------------------
 # the CUDA path
 # ----------------------------------------------------------------------------------------------
 def run_ours(args, wl):
@@ -212,7 +236,7 @@ def run_ours(args, wl):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    wl_rank = dataclasses.replace(wl, seed=wl.seed + 17 * rank)
+    wl_rank = dataclasses.replace(wl, seed=rank_seed(wl.seed, rank))
     peaks = _measured_peaks()
 
     images = make_images(wl_rank, dev)
@@ -265,11 +289,8 @@ def run_ours(args, wl):
     clocks = sampler.stop() if rank == 0 else None
     ctx.poll()
     timers = ctx.timers_read()
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * wl.frames * args.steps / (ms / 1e3)
+    ms = max_over_ranks(ms, world, dev)
+    value = aggregate_frames_per_s(wl.frames, args.steps, world, ms)
 
     # ---- end to end through the host-buffer entry point (same schedule, same weights)
     x_host = [torch.empty(n, d, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
@@ -292,12 +313,9 @@ def run_ours(args, wl):
     ev1.record()
     barrier()
     e2e_ms = max(ev0.elapsed_time(ev1), 1e3 * (time.perf_counter() - t0))  # device span or host wall clock
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
     ctx.poll()
-    e2e_value = world * wl.frames * args.steps / (e2e_ms / 1e3)
+    e2e_value = aggregate_frames_per_s(wl.frames, args.steps, world, e2e_ms)
 
     if rank != 0:
         if world > 1:

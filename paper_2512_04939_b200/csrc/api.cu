@@ -46,7 +46,7 @@ litevggt_status compute_sizes(const litevggt_config& c, Sizes* out) {
   z.frames = c.frames; z.grid_h = c.grid_h; z.grid_w = c.grid_w; z.n_special = c.n_special;
   z.dim = c.dim; z.heads = c.heads;
   const long long p = (long long)c.grid_h * c.grid_w;
-  if (p > 8192) return LITEVGGT_ERR_BAD_CONFIG;
+  if (p > 8192 || c.grid_w > 64) return LITEVGGT_ERR_BAD_CONFIG;  // the Var map kernel stages rows of <= 64 patches
   z.patches = (int)p;
   z.tokens_frame = (int)p + c.n_special;
   z.n_tokens = (long long)c.frames * z.tokens_frame;
@@ -233,6 +233,7 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   const size_t o_keys = c.take<unsigned long long>(cap);
   const size_t o_tmp = c.take<int>(z.n_tokens + 1), o_blk = c.take<int>(2048), o_row = c.take<int>(z.n_tokens);
   const size_t o_qkv = c.take<__nv_bfloat16>(z.n_merged * 3 * z.dim), o_o = c.take<__nv_bfloat16>(z.n_merged * z.dim);
+  const size_t o_vparts = c.take<float>(4 * fp);
   const size_t o_status = c.take<uint32_t>(4);
   Workspace& ws = ctx->ws;
   if (cudaMalloc(&ws.base, c.off) != cudaSuccess) {
@@ -256,6 +257,7 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   ws.row_of = reinterpret_cast<int*>(ws.base + o_row);
   ws.qkv = reinterpret_cast<__nv_bfloat16*>(ws.base + o_qkv);
   ws.attn_o = reinterpret_cast<__nv_bfloat16*>(ws.base + o_o);
+  ws.var_parts = reinterpret_cast<float*>(ws.base + o_vparts);
   ws.status = reinterpret_cast<uint32_t*>(ws.base + o_status);
   if (cudaMemset(ws.base + o_var, 0, o_src - o_var) != cudaSuccess ||
       cudaMemset(ws.status, 0, 16) != cudaSuccess) {
@@ -361,7 +363,7 @@ litevggt_status litevggt_merge_plan(litevggt_ctx* ctx, const void* x, const floa
   cudaError_t e;
   {
     StepTimer t(ctx, 1, s);
-    e = launch_var_map(ctx, xb, ctx->ws.var_map, s, &n);
+    e = launch_var_map(ctx, xb, ctx->ws.var_parts, ctx->ws.var_map, s, &n);
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 2, s);

@@ -23,15 +23,52 @@ grad_map_kernel(const float* __restrict__ images, float* __restrict__ grad, int 
   const int rows = patch + 2;
   const size_t plane = (size_t)h * w;
   const float* img = images + (size_t)f * 3 * plane;
-  for (int idx = threadIdx.x; idx < rows * w; idx += kGradThreads) {
-    const int r = idx / w, xcol = idx - r * w;
-    int y = py * patch - 1 + r;
-    y = y < 0 ? 0 : (y >= h ? h - 1 : y);
-    const size_t o = (size_t)y * w + xcol;
-    const float v = (img[o] + img[plane + o] + img[2 * plane + o]) / 3.0f;
-    grey[r * pitch + xcol + 1] = v;
-    if (xcol == 0) grey[r * pitch] = v;
-    if (xcol == w - 1) grey[r * pitch + w + 1] = v;
+  if ((w & 1) == 0) {
+    // two pixels per load (rows are 8-byte aligned when the width is even), four loads of each
+    // colour plane in flight per thread
+    const int half_w = w >> 1;
+    const int items = rows * half_w;
+    for (int base = threadIdx.x; base < items; base += 4 * kGradThreads) {
+      float2 c0[4], c1[4], c2[4];
+      int rr[4], xx[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int idx = base + u * kGradThreads;
+        const int r = idx < items ? idx / half_w : 0;
+        const int xh = idx < items ? idx - r * half_w : 0;
+        int y = py * patch - 1 + r;
+        y = y < 0 ? 0 : (y >= h ? h - 1 : y);
+        const float2* p = reinterpret_cast<const float2*>(img + (size_t)y * w) + xh;
+        rr[u] = r;
+        xx[u] = 2 * xh;
+        c0[u] = __ldg(p);
+        c1[u] = __ldg(reinterpret_cast<const float2*>(img + plane + (size_t)y * w) + xh);
+        c2[u] = __ldg(reinterpret_cast<const float2*>(img + 2 * plane + (size_t)y * w) + xh);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (base + u * kGradThreads < items) {
+          const float v0 = (c0[u].x + c1[u].x + c2[u].x) / 3.0f;
+          const float v1 = (c0[u].y + c1[u].y + c2[u].y) / 3.0f;
+          float* g = grey + rr[u] * pitch + xx[u] + 1;
+          g[0] = v0;
+          g[1] = v1;
+          if (xx[u] == 0) g[-1] = v0;
+          if (xx[u] == w - 2) g[2] = v1;
+        }
+      }
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < rows * w; idx += kGradThreads) {
+      const int r = idx / w, xcol = idx - r * w;
+      int y = py * patch - 1 + r;
+      y = y < 0 ? 0 : (y >= h ? h - 1 : y);
+      const size_t o = (size_t)y * w + xcol;
+      const float v = (img[o] + img[plane + o] + img[2 * plane + o]) / 3.0f;
+      grey[r * pitch + xcol + 1] = v;
+      if (xcol == 0) grey[r * pitch] = v;
+      if (xcol == w - 1) grey[r * pitch + w + 1] = v;
+    }
   }
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -66,94 +103,145 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 }
 
 // ----------------------------------------------------------------------------------------
-// Var map.  One CTA per (frame, grid row); thread t owns channels 4t..4t+3 and slides a
-// (<=3) x (<=3) window along the row, keeping the three window columns in registers.
-// Two-pass variance in fp32 (mean first, then squared deviations).  Per-position partial
-// sums are reduced over the 256 threads in a fixed order, so the map is deterministic.
-constexpr int kVarThreads = 256;
+// Var map.  One CTA per (frame, grid row, quarter of the channels).  A single thread issues
+// two or three TMA loads - the 256-channel slices of the (clipped) 3 grid rows around the
+// CTA's row - so the whole 57 KB working set of the CTA is in flight at once; with several
+// CTAs per SM that is what keeps HBM busy.  Thread t then owns channels 2(t%128), 2(t%128)+1
+// and slides along its quarter of the row: per column it forms the sums of x - x0 and (x - x0)^2 over the window rows
+// (x0 = the row's first token, per channel, which removes a common offset before squaring),
+// a window is the sum of up to three columns, and the population variance follows as
+// E[d^2] - E[d]^2 in fp32.  The per-position sums over the CTA's 256 channels are reduced in
+// a fixed order and written to this quarter's plane; a second tiny kernel adds the four
+// planes in a fixed order, so the map is deterministic.
+constexpr int kVarThreads = 512;   // 128 channel pairs x 4 segments of the row
+constexpr int kVarSegments = kVarThreads / 128;
+constexpr int kVarChannels = 256;  // per CTA
+constexpr int kVarMaxW = 64;
 
-struct Col3 {
-  float v[3][4];
+struct VarControl {
+  uint64_t bar;
+  uint32_t abort_flag;
 };
-
-__device__ __forceinline__ void load_col(Col3& c, const __nv_bfloat16* row0, int nr, size_t row_pitch, int px) {
-#pragma unroll
-  for (int r = 0; r < 3; ++r) {
-    if (r < nr) {
-      const uint2 raw = *reinterpret_cast<const uint2*>(row0 + r * row_pitch + (size_t)px * 1024);
-      c.v[r][0] = bf16_lo(raw.x);
-      c.v[r][1] = bf16_hi(raw.x);
-      c.v[r][2] = bf16_lo(raw.y);
-      c.v[r][3] = bf16_hi(raw.y);
-    }
-  }
+// dynamic shared memory: [control, 128 B][tile: nr x grid_w x 256 bf16][partial: grid_w x 32 fp32]
+__host__ __device__ inline size_t var_smem_bytes(int grid_w) {
+  return 128 + (size_t)3 * grid_w * kVarChannels * 2 + (size_t)grid_w * 32 * sizeof(float) + 128;
 }
 
 __global__ void __launch_bounds__(kVarThreads)
-var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var, int grid_h, int grid_w, int n_special) {
-  extern __shared__ float partial[];  // [grid_w][256]
-  const int f = blockIdx.y, py = blockIdx.x;
+var_map_kernel(const __grid_constant__ CUtensorMap tmap_x, float* __restrict__ var_parts, int frames, int grid_h,
+               int grid_w, int n_special, uint32_t* status) {
+  extern __shared__ uint8_t var_smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(var_smem_raw) + 127) & ~uintptr_t(127));
+  VarControl* ctrl = reinterpret_cast<VarControl*>(base);
+  uint8_t* tile = base + 128;
+  const uint32_t row_bytes = (uint32_t)grid_w * kVarChannels * 2;  // one grid row of 256-channel slices
+  float* partial = reinterpret_cast<float*>(tile + 3 * (size_t)row_bytes);  // [grid_w][32]
+  const int quarter = blockIdx.x, py = blockIdx.y, f = blockIdx.z;
   const int tokens_frame = grid_h * grid_w + n_special;
   const int r0 = py > 0 ? py - 1 : 0;
   const int r1 = py < grid_h - 1 ? py + 1 : grid_h - 1;
   const int nr = r1 - r0 + 1;
-  const size_t row_pitch = (size_t)grid_w * 1024;
-  const __nv_bfloat16* row0 =
-      x + ((size_t)f * tokens_frame + n_special + (size_t)r0 * grid_w) * 1024 + threadIdx.x * 4;
-  Col3 left, mid, right;
-  load_col(mid, row0, nr, row_pitch, 0);
-  if (grid_w > 1) load_col(right, row0, nr, row_pitch, 1);
-  for (int px = 0; px < grid_w; ++px) {
-    const bool has_l = px > 0, has_r = px < grid_w - 1;
-    const float inv_n = 1.0f / (float)(nr * (1 + (has_l ? 1 : 0) + (has_r ? 1 : 0)));
-    float tot = 0.0f;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float sum = 0.0f;
-#pragma unroll
-      for (int r = 0; r < 3; ++r) {
-        if (r < nr) {
-          sum += mid.v[r][c];
-          if (has_l) sum += left.v[r][c];
-          if (has_r) sum += right.v[r][c];
-        }
-      }
-      const float mu = sum * inv_n;
-      float ss = 0.0f;
-#pragma unroll
-      for (int r = 0; r < 3; ++r) {
-        if (r < nr) {
-          float d = mid.v[r][c] - mu;
-          ss += d * d;
-          if (has_l) { d = left.v[r][c] - mu; ss += d * d; }
-          if (has_r) { d = right.v[r][c] - mu; ss += d * d; }
-        }
-      }
-      tot += ss * inv_n;
-    }
-    partial[px * kVarThreads + threadIdx.x] = tot;
-    left = mid;
-    mid = right;
-    if (px + 2 < grid_w) load_col(right, row0, nr, row_pitch, px + 2);
+  if (threadIdx.x == 0) {
+    mbar_init(&ctrl->bar, 1);
+    ctrl->abort_flag = 0;
+    mbar_fence_init();
   }
   __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int px = warp; px < grid_w; px += kVarThreads / 32) {
-    float acc = 0.0f;
+  if (threadIdx.x == 0) {
+    mbar_expect_tx(&ctrl->bar, row_bytes * nr);
+    for (int r = 0; r < nr; ++r) {
+      const int token = f * tokens_frame + n_special + (r0 + r) * grid_w;
+      tma_load_2d(tile + (size_t)r * row_bytes, &tmap_x, &ctrl->bar, quarter * kVarChannels, token);
+    }
+  }
+  const WaitCtl ctl{&ctrl->abort_flag, status};
+  const bool landed = mbar_wait(&ctrl->bar, 0, ctl);
+  if (!landed && threadIdx.x == 0) {
+    // the copies are still in flight: they must finish before the shared memory is given up
+    const long long t0 = clock64();
+    while (!mbar_try_wait(&ctrl->bar, 0)) {
+      if (clock64() - t0 > kTimeoutCycles) break;
+    }
+  }
+  const int lane = threadIdx.x & 31;
+  if (landed) {
+    const int pair = threadIdx.x & 127, seg = threadIdx.x >> 7;
+    const int seg_len = (grid_w + kVarSegments - 1) / kVarSegments;
+    const int px_begin = seg * seg_len, px_end = min(grid_w, px_begin + seg_len);
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(tile) + pair;  // this thread's channel pair
+    const int pitch = kVarChannels / 2;   // 32-bit words per token slice
+    const int row_words = grid_w * pitch; // per grid row
+    const uint32_t w0 = words[(py - r0) * row_words];
+    const float x0a = bf16_lo(w0), x0b = bf16_hi(w0);
+    // column sums of d and d^2 over the window rows, for the two channels of this thread
+    auto column = [&](int px, float (&s1)[2], float (&s2)[2]) {
+      s1[0] = s1[1] = s2[0] = s2[1] = 0.0f;
+      if (px < 0 || px >= grid_w) return;
 #pragma unroll
-    for (int i = 0; i < kVarThreads / 32; ++i) acc += partial[px * kVarThreads + i * 32 + lane];
+      for (int r = 0; r < 3; ++r) {
+        if (r < nr) {
+          const uint32_t w = words[r * row_words + px * pitch];
+          const float da = bf16_lo(w) - x0a, db = bf16_hi(w) - x0b;
+          s1[0] += da; s1[1] += db;
+          s2[0] = fmaf(da, da, s2[0]); s2[1] = fmaf(db, db, s2[1]);
+        }
+      }
+    };
+    float l1[2], l2[2], m1[2], m2[2], n1[2], n2[2];
+    column(px_begin - 1, l1, l2);
+    column(px_begin, m1, m2);
+    column(px_begin + 1, n1, n2);
+    for (int px = px_begin; px < px_end; ++px) {
+      const int cols = 1 + (px > 0 ? 1 : 0) + (px < grid_w - 1 ? 1 : 0);
+      const float inv_n = 1.0f / (float)(nr * cols);
+      float tot = 0.0f;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const float mean = (l1[c] + m1[c] + n1[c]) * inv_n;
+        const float msq = (l2[c] + m2[c] + n2[c]) * inv_n;
+        tot += fmaxf(fmaf(-mean, mean, msq), 0.0f);
+      }
+      // fixed-order partial reduction over groups of four lanes
+      tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+      tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+      if ((lane & 3) == 0) partial[px * 32 + (pair >> 2)] = tot;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) { l1[c] = m1[c]; l2[c] = m2[c]; m1[c] = n1[c]; m2[c] = n2[c]; }
+      column(px + 2, n1, n2);
+    }
+  }
+  __syncthreads();
+  if (!landed) return;
+  const int warp = threadIdx.x >> 5;
+  float* out = var_parts + ((size_t)quarter * frames + f) * grid_h * grid_w + (size_t)py * grid_w;
+  for (int px = warp; px < grid_w; px += kVarThreads / 32) {
+    float acc = partial[px * 32 + lane];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) var[((size_t)f * grid_h + py) * grid_w + px] = acc / 1024.0f;
+    if (lane == 0) out[px] = acc;
   }
 }
 
-cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var, cudaStream_t s, int* launches) {
+__global__ void var_sum_kernel(const float* __restrict__ parts, float* __restrict__ var, long long count) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) var[i] = (((parts[i] + parts[count + i]) + parts[2 * count + i]) + parts[3 * count + i]) / 1024.0f;
+}
+
+cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var_parts, float* var,
+                           cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
-  const size_t smem = (size_t)z.grid_w * kVarThreads * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  CUtensorMap tmap;
+  if (!make_tmap_bf16_2d_linear(ctx->encode_tiled, &tmap, x, 1024, (uint64_t)z.n_tokens, 1024, kVarChannels,
+                                (uint32_t)z.grid_w))
+    return cudaErrorInvalidValue;
+  const int smem = (int)var_smem_bytes(z.grid_w);
+  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  var_map_kernel<<<dim3(z.grid_h, z.frames), kVarThreads, smem, s>>>(x, var, z.grid_h, z.grid_w, z.n_special);
+  var_map_kernel<<<dim3(4, z.grid_h, z.frames), kVarThreads, smem, s>>>(tmap, var_parts, z.frames, z.grid_h, z.grid_w,
+                                                                        z.n_special, ctx->ws.status);
+  ++*launches;
+  const long long count = (long long)z.frames * z.patches;
+  var_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(var_parts, var, count);
   ++*launches;
   return cudaGetLastError();
 }
