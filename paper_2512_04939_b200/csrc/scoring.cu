@@ -121,6 +121,7 @@ constexpr int kVarMaxW = 64;
 struct VarControl {
   uint64_t bar;
   uint32_t abort_flag;
+  uint32_t landed;
 };
 // dynamic shared memory: [control, 128 B][tile: nr x grid_w x 256 bf16][partial: grid_w x 32 fp32]
 __host__ __device__ inline size_t var_smem_bytes(int grid_w) {
@@ -154,15 +155,22 @@ var_map_kernel(const __grid_constant__ CUtensorMap tmap_x, float* __restrict__ v
       tma_load_2d(tile + (size_t)r * row_bytes, &tmap_x, &ctrl->bar, quarter * kVarChannels, token);
     }
   }
-  const WaitCtl ctl{&ctrl->abort_flag, status};
-  const bool landed = mbar_wait(&ctrl->bar, 0, ctl);
-  if (!landed && threadIdx.x == 0) {
-    // the copies are still in flight: they must finish before the shared memory is given up
-    const long long t0 = clock64();
-    while (!mbar_try_wait(&ctrl->bar, 0)) {
-      if (clock64() - t0 > kTimeoutCycles) break;
+  // Only the issuing thread polls the barrier; everyone else parks at the CTA barrier, which costs
+  // no issue slots (hundreds of polling threads would starve the CTAs that are computing).
+  if (threadIdx.x == 0) {
+    const WaitCtl ctl{&ctrl->abort_flag, status};
+    bool ok = mbar_wait(&ctrl->bar, 0, ctl);
+    if (!ok) {
+      // the copies are still in flight: they must finish before the shared memory is given up
+      const long long t0 = clock64();
+      while (!mbar_try_wait(&ctrl->bar, 0)) {
+        if (clock64() - t0 > kTimeoutCycles) break;
+      }
     }
+    ctrl->landed = ok ? 1u : 0u;
   }
+  __syncthreads();
+  const bool landed = ctrl->landed != 0u;
   const int lane = threadIdx.x & 31;
   if (landed) {
     const int pair = threadIdx.x & 127, seg = threadIdx.x >> 7;
@@ -172,42 +180,57 @@ var_map_kernel(const __grid_constant__ CUtensorMap tmap_x, float* __restrict__ v
     const int pitch = kVarChannels / 2;   // 32-bit words per token slice
     const int row_words = grid_w * pitch; // per grid row
     const uint32_t w0 = words[(py - r0) * row_words];
-    const float x0a = bf16_lo(w0), x0b = bf16_hi(w0);
-    // column sums of d and d^2 over the window rows, for the two channels of this thread
-    auto column = [&](int px, float (&s1)[2], float (&s2)[2]) {
-      s1[0] = s1[1] = s2[0] = s2[1] = 0.0f;
-      if (px < 0 || px >= grid_w) return;
-#pragma unroll
-      for (int r = 0; r < 3; ++r) {
-        if (r < nr) {
-          const uint32_t w = words[r * row_words + px * pitch];
-          const float da = bf16_lo(w) - x0a, db = bf16_hi(w) - x0b;
-          s1[0] += da; s1[1] += db;
-          s2[0] = fmaf(da, da, s2[0]); s2[1] = fmaf(db, db, s2[1]);
-        }
+    const float2 x0 = make_float2(bf16_lo(w0), bf16_hi(w0));
+    const bool three = nr == 3;  // CTA-uniform
+    // column sums of d and d^2 over the window rows, for the two channels of this thread (packed)
+    auto column = [&](int px, float2& s1, float2& s2) {
+      if (px < 0 || px >= grid_w) {
+        s1 = s2 = make_float2(0.0f, 0.0f);
+        return;
+      }
+      const uint32_t* p = words + px * pitch;
+      const uint32_t wa = p[0], wb = p[row_words];
+      const float2 da = make_float2(bf16_lo(wa) - x0.x, bf16_hi(wa) - x0.y);
+      const float2 db = make_float2(bf16_lo(wb) - x0.x, bf16_hi(wb) - x0.y);
+      s1 = __fadd2_rn(da, db);
+      s2 = __ffma2_rn(db, db, __fmul2_rn(da, da));
+      if (three) {
+        const uint32_t wc = p[2 * row_words];
+        const float2 dc = make_float2(bf16_lo(wc) - x0.x, bf16_hi(wc) - x0.y);
+        s1 = __fadd2_rn(s1, dc);
+        s2 = __ffma2_rn(dc, dc, s2);
       }
     };
-    float l1[2], l2[2], m1[2], m2[2], n1[2], n2[2];
-    column(px_begin - 1, l1, l2);
-    column(px_begin, m1, m2);
-    column(px_begin + 1, n1, n2);
-    for (int px = px_begin; px < px_end; ++px) {
-      const int cols = 1 + (px > 0 ? 1 : 0) + (px < grid_w - 1 ? 1 : 0);
-      const float inv_n = 1.0f / (float)(nr * cols);
-      float tot = 0.0f;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const float mean = (l1[c] + m1[c] + n1[c]) * inv_n;
-        const float msq = (l2[c] + m2[c] + n2[c]) * inv_n;
-        tot += fmaxf(fmaf(-mean, mean, msq), 0.0f);
-      }
+    const float inv_edge = 1.0f / (float)(nr * (grid_w > 1 ? 2 : 1)), inv_mid = 1.0f / (float)(nr * 3);
+    // one output position from the three column sums around it
+    auto emit = [&](int px, const float2& a1, const float2& a2, const float2& b1, const float2& b2, const float2& c1,
+                    const float2& c2) {
+      const float inv_n = (px == 0 || px == grid_w - 1) ? inv_edge : inv_mid;
+      const float2 inv2 = make_float2(inv_n, inv_n);
+      const float2 mean = __fmul2_rn(__fadd2_rn(__fadd2_rn(a1, b1), c1), inv2);
+      const float2 msq = __fmul2_rn(__fadd2_rn(__fadd2_rn(a2, b2), c2), inv2);
+      const float2 v = __ffma2_rn(make_float2(-mean.x, -mean.y), mean, msq);
+      float tot = fmaxf(v.x, 0.0f) + fmaxf(v.y, 0.0f);
       // fixed-order partial reduction over groups of four lanes
       tot += __shfl_xor_sync(0xffffffffu, tot, 1);
       tot += __shfl_xor_sync(0xffffffffu, tot, 2);
       if ((lane & 3) == 0) partial[px * 32 + (pair >> 2)] = tot;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) { l1[c] = m1[c]; l2[c] = m2[c]; m1[c] = n1[c]; m2[c] = n2[c]; }
-      column(px + 2, n1, n2);
+    };
+    float2 a1, a2, b1, b2, c1, c2;
+    column(px_begin - 1, a1, a2);
+    column(px_begin, b1, b2);
+    // three positions per trip, so the column sums rotate through fixed registers
+    for (int px = px_begin; px < px_end; px += 3) {
+      column(px + 1, c1, c2);
+      emit(px, a1, a2, b1, b2, c1, c2);
+      if (px + 1 < px_end) {
+        column(px + 2, a1, a2);
+        emit(px + 1, b1, b2, c1, c2, a1, a2);
+      }
+      if (px + 2 < px_end) {
+        column(px + 3, b1, b2);
+        emit(px + 2, c1, c2, a1, a2, b1, b2);
+      }
     }
   }
   __syncthreads();
