@@ -66,6 +66,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Same test, but the hardware may park the thread for up to `ns` nanoseconds while the phase
+// is still open, so a waiting warp does not spend issue slots that computing warps need.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 
 // Per-CTA abort flag (shared memory) plus the context's status word (global memory).
 struct WaitCtl {
@@ -78,16 +91,13 @@ struct WaitCtl {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtl& ctl) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  uint32_t it = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((++it & 31u) == 0u) {
-      if (*ctl.abort_flag != 0u) return false;
-      if (clock64() - t0 > kTimeoutCycles) {
-        *ctl.abort_flag = 1u;
-        atomicOr(ctl.status, kStatusTimeout);
-        return false;
-      }
+    if (mbar_try_wait_parked(bar, parity, 2000u)) return true;  // parks for at most 2 us per try
+    if (*ctl.abort_flag != 0u) return false;
+    if (clock64() - t0 > kTimeoutCycles) {
+      *ctl.abort_flag = 1u;
+      atomicOr(ctl.status, kStatusTimeout);
+      return false;
     }
   }
 }
