@@ -217,15 +217,16 @@ def test_linear(lib, m, k, n):
 def attention_core_bound(qkv, ref_o):
     """Tolerance of the attention core in bf16 arithmetic.  Besides the rounding of the output
     itself (bf16_bound), the probabilities enter the second tensor-core product as bf16, each
-    with a relative error of up to 2^-9, which moves an output by at most
-    2^-9 * sum_i p_i |v_i| / sum_i p_i.  When a few keys dominate a row the two terms are of
+    with a relative error of up to 2^-8 (half an ulp of an 8-bit significand, at the bottom of a
+    binade), which moves an output by at most 2^-8 * sum_i p_i |v_i| / sum_i p_i.  When attention is
+    nearly uniform all probabilities round the same way, so this is a bias, not noise.  When a few keys dominate a row the two terms are of
     the same size, so the second one is part of the bound, evaluated with the oracle on |V|."""
     d = qkv.shape[1] // 3
     abs_v = qkv.copy()
     abs_v[:, 2 * d:] = np.abs(abs_v[:, 2 * d:])
     weighted_abs = O.attention_core(abs_v, heads=16)
     rms = float(np.sqrt(np.mean(ref_o * ref_o)))
-    return bf16_bound(ref_o) + 2.0 ** -9 * float(weighted_abs.max()) / rms
+    return bf16_bound(ref_o) + 2.0 ** -8 * float(weighted_abs.max()) / rms
 
 
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
