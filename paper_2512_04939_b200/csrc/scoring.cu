@@ -8,93 +8,88 @@
 namespace lv {
 
 // ----------------------------------------------------------------------------------------
-// Grad map.  One CTA per (frame, patch row): stages the 16 grey rows it needs (14 + one
-// halo row above and below, replicate padding) in shared memory, then one warp per patch
-// sums the Sobel magnitudes of its 14 x 14 pixels in a fixed order.
+// Grad map.  One CTA per (frame, patch row).  Phase 1: the 16 grey rows it needs (14 + one halo
+// row above and below, replicate padding) are staged in shared memory, one warp per image row,
+// two pixels per load when the width is even.  Phase 2: one thread per pixel column walks down
+// the 16 rows with the separable form of the Sobel pair - per row the horizontal difference
+// r - l and the horizontal smoothing l + 2c + r, kept for the last three rows - and adds up the
+// 14 magnitudes of its column.  Phase 3: one thread per patch adds its 14 column sums.  All sums
+// run in a fixed order.
 constexpr int kGradThreads = 256;
+
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 __global__ void __launch_bounds__(kGradThreads)
 grad_map_kernel(const float* __restrict__ images, float* __restrict__ grad, int grid_h, int grid_w, int patch) {
-  extern __shared__ float grey[];  // [(patch+2)][w+2]
+  extern __shared__ float grey[];  // [(patch+2)][w+2], then [w] column sums
   const int f = blockIdx.y;
   const int py = blockIdx.x;
   const int h = grid_h * patch, w = grid_w * patch;
   const int pitch = w + 2;
   const int rows = patch + 2;
+  float* colsum = grey + rows * pitch;
   const size_t plane = (size_t)h * w;
   const float* img = images + (size_t)f * 3 * plane;
-  if ((w & 1) == 0) {
-    // two pixels per load (rows are 8-byte aligned when the width is even), four loads of each
-    // colour plane in flight per thread
-    const int half_w = w >> 1;
-    const int items = rows * half_w;
-    for (int base = threadIdx.x; base < items; base += 4 * kGradThreads) {
-      float2 c0[4], c1[4], c2[4];
-      int rr[4], xx[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int idx = base + u * kGradThreads;
-        const int r = idx < items ? idx / half_w : 0;
-        const int xh = idx < items ? idx - r * half_w : 0;
-        int y = py * patch - 1 + r;
-        y = y < 0 ? 0 : (y >= h ? h - 1 : y);
-        const float2* p = reinterpret_cast<const float2*>(img + (size_t)y * w) + xh;
-        rr[u] = r;
-        xx[u] = 2 * xh;
-        c0[u] = __ldg(p);
-        c1[u] = __ldg(reinterpret_cast<const float2*>(img + plane + (size_t)y * w) + xh);
-        c2[u] = __ldg(reinterpret_cast<const float2*>(img + 2 * plane + (size_t)y * w) + xh);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r = warp; r < rows; r += kGradThreads / 32) {
+    int y = py * patch - 1 + r;
+    y = y < 0 ? 0 : (y >= h ? h - 1 : y);
+    const float* p0 = img + (size_t)y * w;
+    float* g = grey + r * pitch + 1;
+    if ((w & 1) == 0) {  // rows are 8-byte aligned
+      const float2* q0 = reinterpret_cast<const float2*>(p0);
+      const float2* q1 = reinterpret_cast<const float2*>(p0 + plane);
+      const float2* q2 = reinterpret_cast<const float2*>(p0 + 2 * plane);
+      const int half_w = w >> 1;
+#pragma unroll 4
+      for (int xh = lane; xh < half_w; xh += 32) {
+        const float2 a = __ldg(q0 + xh), b = __ldg(q1 + xh), c = __ldg(q2 + xh);
+        g[2 * xh] = (a.x + b.x + c.x) / 3.0f;
+        g[2 * xh + 1] = (a.y + b.y + c.y) / 3.0f;
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (base + u * kGradThreads < items) {
-          const float v0 = (c0[u].x + c1[u].x + c2[u].x) / 3.0f;
-          const float v1 = (c0[u].y + c1[u].y + c2[u].y) / 3.0f;
-          float* g = grey + rr[u] * pitch + xx[u] + 1;
-          g[0] = v0;
-          g[1] = v1;
-          if (xx[u] == 0) g[-1] = v0;
-          if (xx[u] == w - 2) g[2] = v1;
-        }
-      }
+    } else {
+#pragma unroll 4
+      for (int x = lane; x < w; x += 32) g[x] = (__ldg(p0 + x) + __ldg(p0 + plane + x) + __ldg(p0 + 2 * plane + x)) / 3.0f;
     }
-  } else {
-    for (int idx = threadIdx.x; idx < rows * w; idx += kGradThreads) {
-      const int r = idx / w, xcol = idx - r * w;
-      int y = py * patch - 1 + r;
-      y = y < 0 ? 0 : (y >= h ? h - 1 : y);
-      const size_t o = (size_t)y * w + xcol;
-      const float v = (img[o] + img[plane + o] + img[2 * plane + o]) / 3.0f;
-      grey[r * pitch + xcol + 1] = v;
-      if (xcol == 0) grey[r * pitch] = v;
-      if (xcol == w - 1) grey[r * pitch + w + 1] = v;
+    __syncwarp();
+    if (lane == 0) {
+      g[-1] = g[0];
+      g[w] = g[w - 1];
     }
   }
   __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int npix = patch * patch;
-  for (int px = warp; px < grid_w; px += kGradThreads / 32) {
+  for (int col = threadIdx.x; col < w; col += kGradThreads) {
+    const float* p = grey + col;  // p[0], p[1], p[2] = left, centre, right of this column in row 0
+    float d0 = p[2] - p[0], s0 = fmaf(2.0f, p[1], p[0] + p[2]);
+    p += pitch;
+    float d1 = p[2] - p[0], s1 = fmaf(2.0f, p[1], p[0] + p[2]);
     float acc = 0.0f;
-    for (int i = lane; i < npix; i += 32) {
-      const int r = i / patch, c = i - r * patch;
-      const float* p = grey + (r + 1) * pitch + px * patch + c + 1;  // centre pixel
-      const float tl = p[-pitch - 1], tc = p[-pitch], tr = p[-pitch + 1];
-      const float ml = p[-1], mr = p[1];
-      const float bl = p[pitch - 1], bc = p[pitch], br = p[pitch + 1];
-      const float gx = (tr - tl) + 2.0f * (mr - ml) + (br - bl);
-      const float gy = (bl - tl) + 2.0f * (bc - tc) + (br - tr);
-      acc += sqrtf(gx * gx + gy * gy);
+    for (int r = 0; r < patch; ++r) {
+      p += pitch;
+      const float d2 = p[2] - p[0], s2 = fmaf(2.0f, p[1], p[0] + p[2]);
+      const float gx = fmaf(2.0f, d1, d0 + d2);
+      const float gy = s2 - s0;
+      acc += sqrt_approx(fmaf(gx, gx, gy * gy));
+      d0 = d1; s0 = s1; d1 = d2; s1 = s2;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) grad[((size_t)f * grid_h + py) * grid_w + px] = acc / (float)npix;
+    colsum[col] = acc;
+  }
+  __syncthreads();
+  for (int px = threadIdx.x; px < grid_w; px += kGradThreads) {
+    float acc = 0.0f;
+    for (int c = 0; c < patch; ++c) acc += colsum[px * patch + c];
+    grad[((size_t)f * grid_h + py) * grid_w + px] = acc / (float)(patch * patch);
   }
 }
 
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
   const int patch = ctx->cfg.patch_px;
-  const size_t smem = (size_t)(patch + 2) * (z.grid_w * patch + 2) * sizeof(float);
+  const size_t smem = ((size_t)(patch + 2) * (z.grid_w * patch + 2) + (size_t)z.grid_w * patch) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(grad_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   grad_map_kernel<<<dim3(z.grid_h, z.frames), kGradThreads, smem, s>>>(images, grad, z.grid_h, z.grid_w, patch);
