@@ -234,6 +234,9 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   const size_t o_tmp = c.take<int>(z.n_tokens + 1), o_blk = c.take<int>(2048), o_row = c.take<int>(z.n_tokens);
   const size_t o_qkv = c.take<__nv_bfloat16>(z.n_merged * 3 * z.dim), o_o = c.take<__nv_bfloat16>(z.n_merged * z.dim);
   const size_t o_vparts = c.take<float>(4 * fp);
+  size_t ml_off = 0;
+  const size_t state_bytes = attention_state_bytes(z.n_merged, z.dim, z.heads, &ml_off);
+  const size_t o_state = c.take<uint8_t>((long long)state_bytes);
   const size_t o_status = c.take<uint32_t>(4);
   Workspace& ws = ctx->ws;
   if (cudaMalloc(&ws.base, c.off) != cudaSuccess) {
@@ -258,6 +261,10 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   ws.qkv = reinterpret_cast<__nv_bfloat16*>(ws.base + o_qkv);
   ws.attn_o = reinterpret_cast<__nv_bfloat16*>(ws.base + o_o);
   ws.var_parts = reinterpret_cast<float*>(ws.base + o_vparts);
+  if (state_bytes > 0) {
+    ws.attn_o_state = reinterpret_cast<float*>(ws.base + o_state);
+    ws.attn_ml_state = reinterpret_cast<float*>(ws.base + o_state + ml_off);
+  }
   ws.status = reinterpret_cast<uint32_t*>(ws.base + o_status);
   if (cudaMemset(ws.base + o_var, 0, o_src - o_var) != cudaSuccess ||
       cudaMemset(ws.status, 0, 16) != cudaSuccess) {

@@ -37,6 +37,14 @@
 // for 2^f (relative error 7.5e-5, far below the bf16 rounding of P) and n added into the
 // exponent field.
 //
+// Key chunks.  All CTAs of a head stream the same K/V, but they drift apart, so their combined
+// working set is the head's whole K/V; beyond about a quarter of the L2 that no longer stays
+// resident and every CTA would pull its tiles from HBM (measured: 2.4 TB per launch at 520 K
+// keys).  Long sequences are therefore swept in chunks of at most kFaChunkTiles key tiles, one
+// launch per chunk: a chunk's K/V of one head (32 MiB) stays in L2 while all query blocks pass
+// over it.  Between launches the un-normalised fp32 output rows, the reference maximum and the
+// partial row sums are parked in global memory (a few GB of traffic per launch instead).
+//
 // Online softmax in base 2 with a lazily updated reference maximum: the running output
 // is rescaled only when a row maximum grows by more than 2^8 over the reference (the
 // threads then first wait until the tile's last P V has retired), and the final division
@@ -53,6 +61,10 @@ constexpr int kFaThreads = (kFaSoftmaxWarps + 4) * 32;
 constexpr int kFaTileBytes = 128 * 64 * 2;
 constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 384;
 constexpr float kFaRescaleThreshold = 8.0f;
+#ifndef LV_FA_CHUNK_TILES
+#define LV_FA_CHUNK_TILES 1024
+#endif
+constexpr int kFaChunkTiles = LV_FA_CHUNK_TILES;  // 131072 keys: K and V of one head = 32 MiB
 // Of every 8 consecutive pairs of scores, this many take the polynomial exponential.
 #ifndef LV_FA_POLY_PAIRS
 #define LV_FA_POLY_PAIRS 0
@@ -141,7 +153,8 @@ __device__ __forceinline__ void pair_barrier(int id) {  // the two warps of one 
 
 __global__ void __launch_bounds__(kFaThreads, 1)
 flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
-                       __nv_bfloat16* __restrict__ o, int m_rows, int dim, float scale_log2e, uint32_t* status) {
+                       __nv_bfloat16* __restrict__ o, float* __restrict__ o_state, float* __restrict__ ml_state,
+                       int m_rows, int dim, int tile_begin, int tile_end, float scale_log2e, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_k = smem;
@@ -152,8 +165,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * 256;
   const int head = blockIdx.y;
-  const int n_kv = (m_rows + 127) / 128;
-  const int n_steps = 2 * n_kv;  // step n = key tile n/2, half n%2
+  // this launch covers key tiles [tile_begin, tile_end) of ceil(m_rows / 128); local tile j is
+  // key tile tile_begin + j, step n = local tile n/2, half n%2
+  const int n_kv = tile_end - tile_begin;
+  const int n_steps = 2 * n_kv;
+  const bool first_chunk = tile_begin == 0;
+  const bool last_chunk = tile_end * 128 >= m_rows;
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_ready, kFaSoftmaxWarps);
@@ -196,11 +213,13 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
         const uint32_t phase = (uint32_t)(j / kFaStages) & 1u;
         if (!mbar_wait(&bars->k_empty[stage], phase ^ 1u, ctl)) break;
         mbar_expect_tx(&bars->k_full[stage], kFaTileBytes);
-        tma_load_2d(smem_k + stage * kFaTileBytes, &tmap_qkv, &bars->k_full[stage], dim + head * 64, j * 128);
+        tma_load_2d(smem_k + stage * kFaTileBytes, &tmap_qkv, &bars->k_full[stage], dim + head * 64,
+                    (tile_begin + j) * 128);
         ++k_issued;
         if (!mbar_wait(&bars->v_empty[stage], phase ^ 1u, ctl)) break;
         mbar_expect_tx(&bars->v_full[stage], kFaTileBytes);
-        tma_load_2d(smem_v + stage * kFaTileBytes, &tmap_qkv, &bars->v_full[stage], 2 * dim + head * 64, j * 128);
+        tma_load_2d(smem_v + stage * kFaTileBytes, &tmap_qkv, &bars->v_full[stage], 2 * dim + head * 64,
+                    (tile_begin + j) * 128);
         ++v_issued;
       }
       // every load issued by this thread must have landed before the CTA may exit
@@ -248,7 +267,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192), 1024, 1024);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_ts(o_col, s_col + h * 64 + k * 8, v_desc + 128 * k, idesc_pv, (j | h | k) != 0 ? 1u : 0u);
+            umma_ts(o_col, s_col + h * 64 + k * 8, v_desc + 128 * k, idesc_pv,
+                    (!first_chunk || (j | h | k) != 0) ? 1u : 0u);
           if (last) {
             // no further Q K^T follows whose completion would tell the softmax threads that this
             // P V has retired
@@ -298,6 +318,22 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
         for (int i = 0; i < 16; ++i) qreg[i] = 0u;
       }
       tmem_st16(tmem_base + lane_base + kFaColQ + t * 32 + c * 16, qreg);
+      if (!first_chunk) {
+        // take up this row's running output (this thread's 32 channels) where the last chunk left it
+        uint32_t acc[32];
+        if (row < m_rows) {
+          const uint4* src = reinterpret_cast<const uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 v = src[i];
+            acc[4 * i] = v.x; acc[4 * i + 1] = v.y; acc[4 * i + 2] = v.z; acc[4 * i + 3] = v.w;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = 0u;
+        }
+        tmem_st32(o_addr, acc);
+      }
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
@@ -307,6 +343,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     float m_ref = -INFINITY;  // reference maximum, in log2 units (score * scale * log2 e)
     float2 l_sum2[4] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f),
                         make_float2(0.0f, 0.0f)};
+    // per (row, head): reference maximum and the two column halves' partial row sums
+    float* ml_row = ml_state + ((size_t)(row < m_rows ? row : 0) * (dim / 64) + head) * 4;
+    if (!first_chunk) {
+      m_ref = ml_row[0];
+      l_sum2[0].x = ml_row[1 + c];
+    }
     bool ok = true;
     int pair_syncs = 0;  // both warps of a pair must pass the same number of pair barriers
     for (int n = 0; n < n_steps; ++n) {
@@ -316,7 +358,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       uint32_t s[32];
       tmem_ld32(s_addr + h * 64 + c * 32, s);
       tmem_ld_wait();
-      const int valid = m_rows - n * 64 - c * 32;
+      const int valid = m_rows - (tile_begin * 2 + n) * 64 - c * 32;
       if (valid < 32) {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
@@ -338,7 +380,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       pair_barrier(barrier_id);
       ++pair_syncs;
       const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
-      if (n == 0) {
+      if (first_chunk && n == 0) {
         m_ref = mx_scaled;
       } else {
         const bool grow = mx_scaled > m_ref + kFaRescaleThreshold;
@@ -385,20 +427,29 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     const float l_total = l_own + xchg->row_sum[t][c ^ 1][row_in_tile];
     if (ok && mbar_wait_warp(&bars->o_done[t], 0, ctl)) {
       tc_fence_after();
-      const float inv = 1.0f / l_total;
       uint32_t acc[32];
       tmem_ld32(o_addr, acc);
       tmem_ld_wait();
       if (row < m_rows) {
-        uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
+        if (last_chunk) {
+          const float inv = 1.0f / l_total;
+          uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint4 w;
-          w.x = pack_bf16(__uint_as_float(acc[q * 8 + 0]) * inv, __uint_as_float(acc[q * 8 + 1]) * inv);
-          w.y = pack_bf16(__uint_as_float(acc[q * 8 + 2]) * inv, __uint_as_float(acc[q * 8 + 3]) * inv);
-          w.z = pack_bf16(__uint_as_float(acc[q * 8 + 4]) * inv, __uint_as_float(acc[q * 8 + 5]) * inv);
-          w.w = pack_bf16(__uint_as_float(acc[q * 8 + 6]) * inv, __uint_as_float(acc[q * 8 + 7]) * inv);
-          dst[q] = w;
+          for (int q = 0; q < 4; ++q) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(acc[q * 8 + 0]) * inv, __uint_as_float(acc[q * 8 + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(acc[q * 8 + 2]) * inv, __uint_as_float(acc[q * 8 + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(acc[q * 8 + 4]) * inv, __uint_as_float(acc[q * 8 + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(acc[q * 8 + 6]) * inv, __uint_as_float(acc[q * 8 + 7]) * inv);
+            dst[q] = w;
+          }
+        } else {
+          // park the running state for the next chunk's launch
+          uint4* dst = reinterpret_cast<uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+          if (c == 0) ml_row[0] = m_ref;
+          ml_row[1 + c] = l_own;
         }
       }
     }
@@ -424,10 +475,32 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((m + 255) / 256), (unsigned)ctx->sz.heads);
   const float scale_log2e = 0.125f * 1.4426950408889634f;
-  flash_attention_kernel<<<grid, kFaThreads, kFaSmemBytes, s>>>(tmap, qkv, o, (int)m, dim, scale_log2e,
-                                                                ctx->ws.status);
-  ++*launches;
+  // balanced chunks of at most kFaChunkTiles key tiles; more than one needs the state buffers
+  const int n_tiles = (int)((m + 127) / 128);
+  const int n_chunks = (n_tiles + kFaChunkTiles - 1) / kFaChunkTiles;
+  const int per_chunk = (n_tiles + n_chunks - 1) / n_chunks;
+  if (n_chunks > 1 && (ctx->ws.attn_o_state == nullptr || ctx->ws.attn_ml_state == nullptr)) return cudaErrorInvalidValue;
+  for (int begin = 0; begin < n_tiles; begin += per_chunk) {
+    const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
+    flash_attention_kernel<<<grid, kFaThreads, kFaSmemBytes, s>>>(tmap, qkv, o, ctx->ws.attn_o_state,
+                                                                  ctx->ws.attn_ml_state, (int)m, dim, begin, end,
+                                                                  scale_log2e, ctx->ws.status);
+    ++*launches;
+  }
   return cudaGetLastError();
+}
+
+// Rows of fp32 running output and of {reference maximum, two partial row sums, pad} per head that the
+// chunked sweep parks between launches; zero when m fits one chunk.
+size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset) {
+  const long long n_tiles = (m + 127) / 128;
+  if (n_tiles <= kFaChunkTiles) {
+    if (ml_offset) *ml_offset = 0;
+    return 0;
+  }
+  const size_t o_bytes = (size_t)round_up(m * dim * 4, 256);
+  if (ml_offset) *ml_offset = o_bytes;
+  return o_bytes + (size_t)round_up(m * heads * 16, 256);
 }
 
 }  // namespace lv

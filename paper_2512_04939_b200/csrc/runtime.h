@@ -49,6 +49,8 @@ struct Workspace {
   // attention
   __nv_bfloat16* qkv = nullptr;    // [M, 3D]
   __nv_bfloat16* attn_o = nullptr; // [M, D]
+  float* attn_o_state = nullptr;   // [M, D] running output between key chunks (long sequences only)
+  float* attn_ml_state = nullptr;  // [M, heads, 4] reference maximum and partial row sums
   // whole-layer-from-host staging
   __nv_bfloat16* stage_x = nullptr;   // [N, D]
   __nv_bfloat16* stage_xm = nullptr;  // [M, D]
@@ -150,5 +152,6 @@ cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m
 // attention.cu
 cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long m, __nv_bfloat16* o,
                                    cudaStream_t s, int* launches);
+size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset);
 
 }  // namespace lv
