@@ -33,7 +33,22 @@ import torch
 
 from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
 
+import hashlib
+
 METRIC = "frames/s through merge+global-attn+unmerge (plan refreshed every 6th layer)"
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the attention core per layer on
+# workload C5, summed over the layer's key-chunk launches, from one single-pass ncu capture
+# (profiles/flash_attention_C5_dram.md).  Reported only while the kernel source is the one that was
+# measured.
+ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 20.24e9 + 8.21e9, "kernel_sha256": "aebbf49d8b710d85ba540fd6c0553fefcfc30eda9f410f03a0e5dcd1d81e7b1d"}
+
+
+def _attention_source_hash() -> str:
+    h = hashlib.sha256()
+    for name in ("attention.cu", "common.cuh"):
+        with open(os.path.join(ROOT, "paper_2512_04939_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 UNIT = "frames/s"
 CPU_SAMPLE_FRAMES = 16
 
@@ -363,9 +378,14 @@ def run_ours(args, wl):
         "gpu_launches": launches,
         "roofline": {"kernel": "flash_attention_kernel", "bound": "tensor", "achieved": att_tflops,
                      "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
-                     "frac": att_tflops / peaks["bf16_sustained"], "traffic": None,
+                     "frac": att_tflops / peaks["bf16_sustained"],
+                     "traffic": (ATTENTION_TRAFFIC_C5["bytes_per_layer"]
+                                 if wl.name == "C5" and _attention_source_hash() == ATTENTION_TRAFFIC_C5["kernel_sha256"]
+                                 else None),
+                     "traffic_unit": "bytes per layer (all key-chunk launches of one attention core)",
                      "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
-                     "flops_per_launch": att_flops, "ms_per_launch": att_ms / max(att_n, 1)},
+                     "flops_per_launch": att_flops, "ms_per_launch": att_ms / max(att_n, 1),
+                     "launch": "one attention core = the key-chunk launches of one layer, timed as a group"},
         "breakdown": breakdown,
         "cpu_baseline": cpu,
     }
