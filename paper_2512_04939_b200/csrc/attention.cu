@@ -151,6 +151,8 @@ __device__ __forceinline__ void pair_barrier(int id) {  // the two warps of one 
   asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
 }
 
+// kFirst / kLast: this launch holds the first / the last key chunk of the sweep.
+template <bool kFirst, bool kLast>
 __global__ void __launch_bounds__(kFaThreads, 1)
 flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_state, float* __restrict__ ml_state,
@@ -169,8 +171,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   // key tile tile_begin + j, step n = local tile n/2, half n%2
   const int n_kv = tile_end - tile_begin;
   const int n_steps = 2 * n_kv;
-  const bool first_chunk = tile_begin == 0;
-  const bool last_chunk = tile_end * 128 >= m_rows;
+  constexpr bool first_chunk = kFirst;
+  constexpr bool last_chunk = kLast;
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_ready, kFaSoftmaxWarps);
@@ -344,8 +346,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     float2 l_sum2[4] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f),
                         make_float2(0.0f, 0.0f)};
     // per (row, head): reference maximum and the two column halves' partial row sums
-    float* ml_row = ml_state + ((size_t)(row < m_rows ? row : 0) * (dim / 64) + head) * 4;
     if (!first_chunk) {
+      const float* ml_row = ml_state + ((size_t)(row < m_rows ? row : 0) * (dim / 64) + head) * 4;
       m_ref = ml_row[0];
       l_sum2[0].x = ml_row[1 + c];
     }
@@ -448,6 +450,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           uint4* dst = reinterpret_cast<uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i) dst[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+          float* ml_row = ml_state + ((size_t)row * (dim / 64) + head) * 4;
           if (c == 0) ml_row[0] = m_ref;
           ml_row[1 + c] = l_own;
         }
@@ -470,9 +473,15 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   CUtensorMap tmap;
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap, qkv, (uint64_t)3 * dim, (uint64_t)m, (uint64_t)3 * dim, 64, 128))
     return cudaErrorInvalidValue;
-  cudaError_t e =
-      cudaFuncSetAttribute(flash_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmemBytes);
-  if (e != cudaSuccess) return e;
+  using Kernel = void (*)(const CUtensorMap, const __nv_bfloat16*, __nv_bfloat16*, float*, float*, int, int, int, int,
+                          float, uint32_t*);
+  const Kernel kernels[2][2] = {{flash_attention_kernel<false, false>, flash_attention_kernel<false, true>},
+                                {flash_attention_kernel<true, false>, flash_attention_kernel<true, true>}};
+  for (int a = 0; a < 2; ++a)
+    for (int b = 0; b < 2; ++b) {
+      cudaError_t e = cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmemBytes);
+      if (e != cudaSuccess) return e;
+    }
   const dim3 grid((unsigned)((m + 255) / 256), (unsigned)ctx->sz.heads);
   const float scale_log2e = 0.125f * 1.4426950408889634f;
   // balanced chunks of at most kFaChunkTiles key tiles; more than one needs the state buffers
@@ -482,9 +491,9 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   if (n_chunks > 1 && (ctx->ws.attn_o_state == nullptr || ctx->ws.attn_ml_state == nullptr)) return cudaErrorInvalidValue;
   for (int begin = 0; begin < n_tiles; begin += per_chunk) {
     const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
-    flash_attention_kernel<<<grid, kFaThreads, kFaSmemBytes, s>>>(tmap, qkv, o, ctx->ws.attn_o_state,
-                                                                  ctx->ws.attn_ml_state, (int)m, dim, begin, end,
-                                                                  scale_log2e, ctx->ws.status);
+    kernels[begin == 0][end == n_tiles]<<<grid, kFaThreads, kFaSmemBytes, s>>>(
+        tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, (int)m, dim, begin, end, scale_log2e,
+        ctx->ws.status);
     ++*launches;
   }
   return cudaGetLastError();
