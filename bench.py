@@ -402,8 +402,15 @@ def main():
     ap.add_argument("--workload", default="C5", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--interval", type=int, default=None,
+                    help="recompute the merge plan every this many layers (default: the workload's, 6); "
+                         "with --steps 24 this reproduces the paper's recompute-interval ablation")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
+    if args.interval is not None:
+        if args.interval < 1:
+            ap.error("--interval must be >= 1")
+        wl = dataclasses.replace(wl, recompute_interval=args.interval)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -154,6 +154,28 @@ litevggt_status litevggt_global_attn_static(const void* x_merged, int64_t m, con
                                             const void* b_qkv, const void* w_o, const void* b_o,
                                             void* y_merged, uint32_t* device_status, void* stream);
 
+/* The other sub-layers of an aggregator block (Sec. 3.1: the aggregator alternates frame-wise and
+ * global self-attention; pre-norm transformer blocks with an MLP of ratio 4 are the reading taken).
+ * They run at the full length N, outside the merged path.  Their workspace (N x 4D bf16 plus 1 GiB)
+ * is allocated on the first of these calls.
+ *
+ * LayerNorm over the D channels of each row: y = (x - mean) / sqrt(var + eps) * gamma + beta with
+ * the population variance.  x, out: dev bf16 [rows, D]; gamma, beta: dev bf16 [D]. */
+litevggt_status litevggt_layernorm(litevggt_ctx* ctx, const void* x, int64_t rows, const void* gamma, const void* beta,
+                                   float eps, void* out, void* stream);
+
+/* Frame-local self-attention: the same attention layer as litevggt_global_attn applied to every
+ * frame's T = P + S tokens separately (Sec. 3.1), y = residual + attn(x) (residual may be NULL).
+ * x, residual, y: dev bf16 [N, D]; weights as in litevggt_global_attn. */
+litevggt_status litevggt_frame_attn(litevggt_ctx* ctx, const void* x, const void* w_qkv, const void* b_qkv,
+                                    const void* w_o, const void* b_o, const void* residual, void* y, void* stream);
+
+/* Transformer MLP: y = residual + gelu(x w1^T + b1) w2^T + b2 with the exact (erf) GELU.
+ * x, residual (nullable), y: dev bf16 [rows, D], rows <= N; w1: dev bf16 [4D, D]; b1: dev bf16 [4D] or
+ * NULL; w2: dev bf16 [D, 4D]; b2: dev bf16 [D] or NULL. */
+litevggt_status litevggt_mlp(litevggt_ctx* ctx, const void* x, int64_t rows, const void* w1, const void* b1,
+                             const void* w2, const void* b2, const void* residual, void* y, void* stream);
+
 /* Unmerge (Sec. 3.4, "Token Unmerging"): out_i = y'[dst_of[i]] (+ residual_i).
  * y_merged: dev bf16 [M,D];  residual: dev bf16 [N,D] or NULL;  out: dev bf16 [N,D]. */
 litevggt_status litevggt_unmerge(litevggt_ctx* ctx, const litevggt_plan* plan, const void* y_merged,
@@ -206,7 +228,8 @@ litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
 /* Device-time stopwatches.  Each step of the path is bracketed by CUDA events recorded on
  * the launching stream: which = 0 grad map, 1 var map, 2 partition + token lists, 3 cosine
  * matching (pack + GEMM/argmax), 4 selection + index build, 5 merge, 6 qkv projection,
- * 7 attention core, 8 output projection, 9 unmerge.  litevggt_timers_reset forgets all
+ * 7 attention core, 8 output projection, 9 unmerge, 10 LayerNorm, 11 frame-local attention layer,
+ * 12 MLP.  litevggt_timers_reset forgets all
  * records; litevggt_timer_read synchronises on the recorded events and returns the summed
  * device time (ms) and the number of records (at most 64 are kept per step). */
 litevggt_status litevggt_timers_reset(litevggt_ctx* ctx);

@@ -299,6 +299,44 @@ def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024
 
 
 # --------------------------------------------------------------------------------------
+# the other sub-layers of an aggregator block (Sec. 3.1)
+# --------------------------------------------------------------------------------------
+def layernorm(x, gamma, beta, eps=1e-6):
+    """LayerNorm over the channels of each row, population variance (the pre-norm of the
+    transformer blocks the aggregator is built from, Sec. 3.1)."""
+    x = np.asarray(x, dtype=np.float64)
+    mu = x.mean(axis=1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps) * np.asarray(gamma, dtype=np.float64) + np.asarray(beta, dtype=np.float64)
+
+
+def gelu(x):
+    """Exact GELU: x * Phi(x), Phi the standard normal distribution function."""
+    from math import erf, sqrt
+    x = np.asarray(x, dtype=np.float64)
+    return 0.5 * x * (1.0 + np.vectorize(erf)(x / sqrt(2.0)))
+
+
+def mlp(x, w1, b1, w2, b2, residual=None):
+    """Transformer MLP of ratio 4: gelu(x w1^T + b1) w2^T + b2 (+ residual)."""
+    y = linear(gelu(linear(x, w1, b1)), w2, b2)
+    if residual is not None:
+        y = y + np.asarray(residual, dtype=np.float64)
+    return y
+
+
+def frame_attention(x, frames, w_qkv, b_qkv, w_o, b_o, heads=16, residual=None):
+    """Frame-wise self-attention (Sec. 3.1): every frame's tokens attend only to the tokens of the
+    same frame; the layer itself is the one of global_attention."""
+    x = np.asarray(x, dtype=np.float64)
+    t = x.shape[0] // frames
+    y = np.concatenate([global_attention(x[f * t:(f + 1) * t], w_qkv, b_qkv, w_o, b_o, heads) for f in range(frames)])
+    if residual is not None:
+        y = y + np.asarray(residual, dtype=np.float64)
+    return y
+
+
+# --------------------------------------------------------------------------------------
 # index cache
 # --------------------------------------------------------------------------------------
 def should_refresh(global_layer_idx, recompute_interval=6):

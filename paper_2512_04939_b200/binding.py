@@ -62,6 +62,9 @@ def load_library():
         "litevggt_global_attn": [vp, vp, i64, vp, vp, vp, vp, vp, vp],
         "litevggt_global_attn_static": [vp, i64, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_unmerge": [vp, vp, vp, vp, vp, vp],
+        "litevggt_layernorm": [vp, vp, i64, vp, vp, C.c_float, vp, vp],
+        "litevggt_frame_attn": [vp, vp, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_mlp": [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_global_layer_host": [vp, P(vp), vp, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_timers_reset": [vp],
         "litevggt_timer_read": [vp, C.c_int, P(C.c_float), P(i32)],
@@ -232,6 +235,30 @@ class LiteVGGT:
                "global_layer_host")
         return plan if plan is not None else Plan(self, h)
 
+    def layernorm(self, x, gamma, beta, eps=1e-6, out=None) -> torch.Tensor:
+        assert x.dtype == torch.bfloat16 and x.shape[1] == self.dim
+        if out is None:
+            out = torch.empty_like(x)
+        _check(self.lib.litevggt_layernorm(self.handle, _ptr(x), x.shape[0], _ptr(gamma), _ptr(beta), eps, _ptr(out),
+                                           _stream()), "layernorm")
+        return out
+
+    def frame_attn(self, x, w_qkv, b_qkv, w_o, b_o, residual=None, out=None) -> torch.Tensor:
+        assert x.dtype == torch.bfloat16 and x.shape == (self.n_tokens, self.dim)
+        if out is None:
+            out = torch.empty_like(x)
+        _check(self.lib.litevggt_frame_attn(self.handle, _ptr(x), _ptr(w_qkv), _ptr(b_qkv), _ptr(w_o), _ptr(b_o),
+                                            _ptr(residual), _ptr(out), _stream()), "frame_attn")
+        return out
+
+    def mlp(self, x, w1, b1, w2, b2, residual=None, out=None) -> torch.Tensor:
+        assert x.dtype == torch.bfloat16 and x.shape[1] == self.dim
+        if out is None:
+            out = torch.empty_like(x)
+        _check(self.lib.litevggt_mlp(self.handle, _ptr(x), x.shape[0], _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2),
+                                     _ptr(residual), _ptr(out), _stream()), "mlp")
+        return out
+
     def linear(self, a, w, bias=None) -> torch.Tensor:
         m, k = a.shape
         n = w.shape[0]
@@ -280,7 +307,7 @@ class LiteVGGT:
         return torch.as_tensor(view, device=self.device).view(torch.bfloat16).clone()
 
     TIMER_NAMES = ("grad_map", "var_map", "partition", "match", "index_build", "merge", "qkv_proj",
-                   "attention", "out_proj", "unmerge")
+                   "attention", "out_proj", "unmerge", "layernorm", "frame_attn", "mlp")
 
     def timers_reset(self):
         _check(self.lib.litevggt_timers_reset(self.handle), "timers_reset")

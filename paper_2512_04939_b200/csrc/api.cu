@@ -177,6 +177,26 @@ litevggt_status ensure_staging(litevggt_ctx* ctx) {
   return LITEVGGT_OK;
 }
 
+litevggt_status ensure_block_ws(litevggt_ctx* ctx) {
+  if (ctx->ws.blk_qkv != nullptr) return LITEVGGT_OK;
+  const Sizes& z = ctx->sz;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LITEVGGT_ERR_CUDA;
+  const size_t qkv = (size_t)round_up(z.n_tokens * 3 * z.dim * 2, 256), o = (size_t)round_up(z.n_tokens * z.dim * 2, 256);
+  const long long hid_rows = z.n_tokens < kMlpChunkRows ? z.n_tokens : kMlpChunkRows;
+  const size_t hid = (size_t)round_up(hid_rows * 4 * z.dim * 2, 256);
+  uint8_t* base = nullptr;
+  if (cudaMalloc(&base, qkv + o + hid) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return LITEVGGT_ERR_ALLOC;
+  }
+  ctx->ws.blk_qkv = reinterpret_cast<__nv_bfloat16*>(base);
+  ctx->ws.blk_o = reinterpret_cast<__nv_bfloat16*>(base + qkv);
+  ctx->ws.blk_hidden = reinterpret_cast<__nv_bfloat16*>(base + qkv + o);
+  ctx->ws.bytes += qkv + o + hid;
+  return LITEVGGT_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -323,6 +343,7 @@ litevggt_status litevggt_destroy(litevggt_ctx* ctx) {
         cudaEventDestroy(ctx->timers.stop[w][i]);
       }
   if (ctx->ws.stage_x != nullptr) cudaFree(ctx->ws.stage_x);
+  if (ctx->ws.blk_qkv != nullptr) cudaFree(ctx->ws.blk_qkv);
   if (ctx->ws.base != nullptr) cudaFree(ctx->ws.base);
   (void)cudaGetLastError();
   ctx->magic = 0;
@@ -450,12 +471,89 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 7, s);
-    e = launch_flash_attention(ctx, ctx->ws.qkv, m, ctx->ws.attn_o, s, &n);
+    e = launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 8, s);
     e = launch_linear(ctx, ctx->ws.attn_o, m, d, static_cast<const __nv_bfloat16*>(w_o), d,
                       static_cast<const __nv_bfloat16*>(b_o), static_cast<__nv_bfloat16*>(y_merged), s, &n);
+  }
+  bump(ctx, n);
+  return cuda_status(e);
+}
+
+litevggt_status litevggt_layernorm(litevggt_ctx* ctx, const void* x, int64_t rows, const void* gamma, const void* beta,
+                                   float eps, void* out, void* stream) {
+  if (!ctx_ok(ctx) || x == nullptr || gamma == nullptr || beta == nullptr || out == nullptr) return LITEVGGT_ERR_NULL;
+  if (rows < 0 || !(eps > 0.0f)) return LITEVGGT_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(gamma) || !aligned16(beta) || !aligned16(out)) return LITEVGGT_ERR_ALIGN;
+  int n = 0;
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 10, (cudaStream_t)stream);
+    e = launch_layernorm(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(gamma),
+                         static_cast<const __nv_bfloat16*>(beta), static_cast<__nv_bfloat16*>(out), rows, eps,
+                         (cudaStream_t)stream, &n);
+  }
+  bump(ctx, n);
+  return cuda_status(e);
+}
+
+litevggt_status litevggt_frame_attn(litevggt_ctx* ctx, const void* x, const void* w_qkv, const void* b_qkv,
+                                    const void* w_o, const void* b_o, const void* residual, void* y, void* stream) {
+  if (!ctx_ok(ctx) || x == nullptr || w_qkv == nullptr || w_o == nullptr || y == nullptr) return LITEVGGT_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(w_o) || !aligned16(y) ||
+      (b_qkv != nullptr && !aligned16(b_qkv)) || (b_o != nullptr && !aligned16(b_o)) ||
+      (residual != nullptr && !aligned16(residual)))
+    return LITEVGGT_ERR_ALIGN;
+  litevggt_status st = ensure_block_ws(ctx);
+  if (st != LITEVGGT_OK) return st;
+  const Sizes& z = ctx->sz;
+  const int d = z.dim;
+  cudaStream_t s = (cudaStream_t)stream;
+  int n = 0;
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 11, s);
+    e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x), z.n_tokens, d, static_cast<const __nv_bfloat16*>(w_qkv),
+                      3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.blk_qkv, s, &n);
+    if (e == cudaSuccess) e = launch_flash_attention(ctx, ctx->ws.blk_qkv, z.tokens_frame, z.frames, ctx->ws.blk_o, s, &n);
+    if (e == cudaSuccess)
+      e = launch_linear_mlp(ctx, ctx->ws.blk_o, z.n_tokens, d, static_cast<const __nv_bfloat16*>(w_o), d,
+                            static_cast<const __nv_bfloat16*>(b_o), 0, static_cast<const __nv_bfloat16*>(residual),
+                            static_cast<__nv_bfloat16*>(y), s, &n);
+  }
+  bump(ctx, n);
+  return cuda_status(e);
+}
+
+litevggt_status litevggt_mlp(litevggt_ctx* ctx, const void* x, int64_t rows, const void* w1, const void* b1,
+                             const void* w2, const void* b2, const void* residual, void* y, void* stream) {
+  if (!ctx_ok(ctx) || x == nullptr || w1 == nullptr || w2 == nullptr || y == nullptr) return LITEVGGT_ERR_NULL;
+  if (rows < 0 || rows > ctx->sz.n_tokens) return LITEVGGT_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(w1) || !aligned16(w2) || !aligned16(y) || (b1 != nullptr && !aligned16(b1)) ||
+      (b2 != nullptr && !aligned16(b2)) || (residual != nullptr && !aligned16(residual)))
+    return LITEVGGT_ERR_ALIGN;
+  litevggt_status st = ensure_block_ws(ctx);
+  if (st != LITEVGGT_OK) return st;
+  const int d = ctx->sz.dim;
+  cudaStream_t s = (cudaStream_t)stream;
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  const __nv_bfloat16* rb = static_cast<const __nv_bfloat16*>(residual);
+  __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(y);
+  int n = 0;
+  cudaError_t e = cudaSuccess;
+  {
+    StepTimer t(ctx, 12, s);
+    for (long long r0 = 0; r0 < rows && e == cudaSuccess; r0 += kMlpChunkRows) {
+      const long long nr = rows - r0 < kMlpChunkRows ? rows - r0 : kMlpChunkRows;
+      e = launch_linear_mlp(ctx, xb + r0 * d, nr, d, static_cast<const __nv_bfloat16*>(w1), 4 * d,
+                            static_cast<const __nv_bfloat16*>(b1), 1, nullptr, ctx->ws.blk_hidden, s, &n);
+      if (e == cudaSuccess)
+        e = launch_linear_mlp(ctx, ctx->ws.blk_hidden, nr, 4 * d, static_cast<const __nv_bfloat16*>(w2), d,
+                              static_cast<const __nv_bfloat16*>(b2), 0, rb != nullptr ? rb + r0 * d : nullptr,
+                              yb + r0 * d, s, &n);
+    }
   }
   bump(ctx, n);
   return cuda_status(e);

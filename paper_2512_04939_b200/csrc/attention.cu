@@ -156,7 +156,7 @@ template <bool kFirst, bool kLast>
 __global__ void __launch_bounds__(kFaThreads, 1)
 flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_state, float* __restrict__ ml_state,
-                       int m_rows, int dim, int tile_begin, int tile_end, float scale_log2e, uint32_t* status) {
+                       int seq_len, int dim, int tile_begin, int tile_end, float scale_log2e, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_k = smem;
@@ -165,9 +165,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   FaBarriers* bars = reinterpret_cast<FaBarriers*>(xchg + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q0 = blockIdx.x * 256;
+  // blockIdx.z selects one of the independent sequences of seq_len rows laid back to back (the
+  // global layer has one; a frame-local layer has one per frame)
+  const int row_base = blockIdx.z * seq_len;
+  const int q0 = blockIdx.x * 256;  // within the sequence
   const int head = blockIdx.y;
-  // this launch covers key tiles [tile_begin, tile_end) of ceil(m_rows / 128); local tile j is
+  // this launch covers key tiles [tile_begin, tile_end) of ceil(seq_len / 128); local tile j is
   // key tile tile_begin + j, step n = local tile n/2, half n%2
   const int n_kv = tile_end - tile_begin;
   const int n_steps = 2 * n_kv;
@@ -216,12 +219,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
         if (!mbar_wait(&bars->k_empty[stage], phase ^ 1u, ctl)) break;
         mbar_expect_tx(&bars->k_full[stage], kFaTileBytes);
         tma_load_2d(smem_k + stage * kFaTileBytes, &tmap_qkv, &bars->k_full[stage], dim + head * 64,
-                    (tile_begin + j) * 128);
+                    row_base + (tile_begin + j) * 128);
         ++k_issued;
         if (!mbar_wait(&bars->v_empty[stage], phase ^ 1u, ctl)) break;
         mbar_expect_tx(&bars->v_full[stage], kFaTileBytes);
         tma_load_2d(smem_v + stage * kFaTileBytes, &tmap_qkv, &bars->v_full[stage], 2 * dim + head * 64,
-                    (tile_begin + j) * 128);
+                    row_base + (tile_begin + j) * 128);
         ++v_issued;
       }
       // every load issued by this thread must have landed before the CTA may exit
@@ -302,13 +305,15 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     const int barrier_id = 1 + t * 4 + (int)quarter;
     const int row_in_tile = (int)quarter * 32 + lane;
     const uint32_t lane_base = (quarter * 32u) << 16;
-    const int row = q0 + t * 128 + row_in_tile;
+    const int row_local = q0 + t * 128 + row_in_tile;
+    const bool row_live = row_local < seq_len;
+    const int row = row_base + row_local;  // global row of qkv / o
     const uint32_t s_addr = tmem_base + lane_base + kFaColS + t * 128;
     const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * 64 + c * 32;
     {
       // this thread's half (32 channels) of its query row goes to tensor memory as it is
       uint32_t qreg[16];
-      if (row < m_rows) {
+      if (row_live) {
         const uint4* src = reinterpret_cast<const uint4*>(qkv + (size_t)row * 3 * dim + head * 64 + c * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -323,7 +328,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       if (!first_chunk) {
         // take up this row's running output (this thread's 32 channels) where the last chunk left it
         uint32_t acc[32];
-        if (row < m_rows) {
+        if (row_live) {
           const uint4* src = reinterpret_cast<const uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -347,7 +352,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
                         make_float2(0.0f, 0.0f)};
     // per (row, head): reference maximum and the two column halves' partial row sums
     if (!first_chunk) {
-      const float* ml_row = ml_state + ((size_t)(row < m_rows ? row : 0) * (dim / 64) + head) * 4;
+      const float* ml_row = ml_state + ((size_t)(row_live ? row : 0) * (dim / 64) + head) * 4;
       m_ref = ml_row[0];
       l_sum2[0].x = ml_row[1 + c];
     }
@@ -360,7 +365,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       uint32_t s[32];
       tmem_ld32(s_addr + h * 64 + c * 32, s);
       tmem_ld_wait();
-      const int valid = m_rows - (tile_begin * 2 + n) * 64 - c * 32;
+      const int valid = seq_len - (tile_begin * 2 + n) * 64 - c * 32;
       if (valid < 32) {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
@@ -432,7 +437,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       uint32_t acc[32];
       tmem_ld32(o_addr, acc);
       tmem_ld_wait();
-      if (row < m_rows) {
+      if (row_live) {
         if (last_chunk) {
           const float inv = 1.0f / l_total;
           uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
@@ -466,12 +471,13 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   }
 }
 
-cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long m, __nv_bfloat16* o,
-                                   cudaStream_t s, int* launches) {
-  if (m == 0) return cudaSuccess;
+cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long seq_len, int n_seq,
+                                   __nv_bfloat16* o, cudaStream_t s, int* launches) {
+  if (seq_len == 0 || n_seq == 0) return cudaSuccess;
   const int dim = ctx->sz.dim;
+  const long long rows = seq_len * n_seq;
   CUtensorMap tmap;
-  if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap, qkv, (uint64_t)3 * dim, (uint64_t)m, (uint64_t)3 * dim, 64, 128))
+  if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap, qkv, (uint64_t)3 * dim, (uint64_t)rows, (uint64_t)3 * dim, 64, 128))
     return cudaErrorInvalidValue;
   using Kernel = void (*)(const CUtensorMap, const __nv_bfloat16*, __nv_bfloat16*, float*, float*, int, int, int, int,
                           float, uint32_t*);
@@ -482,17 +488,19 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
       cudaError_t e = cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmemBytes);
       if (e != cudaSuccess) return e;
     }
-  const dim3 grid((unsigned)((m + 255) / 256), (unsigned)ctx->sz.heads);
+  const dim3 grid((unsigned)((seq_len + 255) / 256), (unsigned)ctx->sz.heads, (unsigned)n_seq);
   const float scale_log2e = 0.125f * 1.4426950408889634f;
-  // balanced chunks of at most kFaChunkTiles key tiles; more than one needs the state buffers
-  const int n_tiles = (int)((m + 127) / 128);
+  // balanced chunks of at most kFaChunkTiles key tiles; more than one needs the state buffers (which
+  // are sized for the single long sequence of the global layer)
+  const int n_tiles = (int)((seq_len + 127) / 128);
   const int n_chunks = (n_tiles + kFaChunkTiles - 1) / kFaChunkTiles;
   const int per_chunk = (n_tiles + n_chunks - 1) / n_chunks;
-  if (n_chunks > 1 && (ctx->ws.attn_o_state == nullptr || ctx->ws.attn_ml_state == nullptr)) return cudaErrorInvalidValue;
+  if (n_chunks > 1 && (n_seq != 1 || ctx->ws.attn_o_state == nullptr || ctx->ws.attn_ml_state == nullptr))
+    return cudaErrorInvalidValue;
   for (int begin = 0; begin < n_tiles; begin += per_chunk) {
     const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
     kernels[begin == 0][end == n_tiles]<<<grid, kFaThreads, kFaSmemBytes, s>>>(
-        tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, (int)m, dim, begin, end, scale_log2e,
+        tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, (int)seq_len, dim, begin, end, scale_log2e,
         ctx->ws.status);
     ++*launches;
   }

@@ -108,7 +108,7 @@ extern "C" litevggt_status litevggt_global_attn_static(const void* x_merged, int
   cudaError_t e = lv::launch_linear(&local, static_cast<const __nv_bfloat16*>(x_merged), m, kStaticDim,
                                     static_cast<const __nv_bfloat16*>(w_qkv), 3 * kStaticDim,
                                     static_cast<const __nv_bfloat16*>(b_qkv), qkv, s, &n);
-  if (e == cudaSuccess) e = lv::launch_flash_attention(&local, qkv, m, o, s, &n);
+  if (e == cudaSuccess) e = lv::launch_flash_attention(&local, qkv, m, 1, o, s, &n);
   if (e == cudaSuccess)
     e = lv::launch_linear(&local, o, m, kStaticDim, static_cast<const __nv_bfloat16*>(w_o), kStaticDim,
                           static_cast<const __nv_bfloat16*>(b_o), static_cast<__nv_bfloat16*>(y_merged), s, &n);

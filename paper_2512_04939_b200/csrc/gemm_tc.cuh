@@ -235,6 +235,63 @@ struct LinearEpilogue {
   }
 };
 
+// Epilogue of the MLP layers: out[row, col] = bf16(act(acc + bias[col]) + residual[row, col]) with
+// act = exact GELU (0.5 x (1 + erf(x / sqrt 2))) or the identity, residual optional.
+struct MlpEpilogue {
+  struct State {};
+  __nv_bfloat16* out;
+  const __nv_bfloat16* bias;      // may be null
+  const __nv_bfloat16* residual;  // may be null, same shape and pitch as out
+  int m_rows;
+  int n_cols;
+  long long ld_out;
+  int gelu;
+
+  __device__ __forceinline__ void begin(State&, int) const {}
+  __device__ __forceinline__ void finish(State&, int) const {}
+  __device__ __forceinline__ void consume(State&, int row, int col0, const uint32_t (&acc)[32]) const {
+    if (row >= m_rows || col0 >= n_cols) return;
+    float v[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
+    if (bias != nullptr) {
+      const uint4* bp = reinterpret_cast<const uint4*>(bias + col0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 b = bp[q];
+        const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          v[q * 8 + 2 * i] += bf16_lo(bw[i]);
+          v[q * 8 + 2 * i + 1] += bf16_hi(bw[i]);
+        }
+      }
+    }
+    if (gelu) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = 0.5f * v[i] * (1.0f + erff(v[i] * 0.70710678118654752f));
+    }
+    if (residual != nullptr) {
+      const uint4* rp = reinterpret_cast<const uint4*>(residual + (long long)row * ld_out + col0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 r = rp[q];
+        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          v[q * 8 + 2 * i] += bf16_lo(rw[i]);
+          v[q * 8 + 2 * i + 1] += bf16_hi(rw[i]);
+        }
+      }
+    }
+    uint4* op = reinterpret_cast<uint4*>(out + (long long)row * ld_out + col0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      op[q] = make_uint4(pack_bf16(v[q * 8], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+                         pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+  }
+};
+
 // Epilogue: running argmax over columns of acc[row, col] * inv_norm_b[col]; at the end
 // best_idx[row] = col_ids[argmax], best_val[row] = max * inv_norm_a[row].
 // Columns are visited in ascending order and only a strictly larger value replaces the

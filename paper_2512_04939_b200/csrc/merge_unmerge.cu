@@ -126,6 +126,67 @@ unmerge_kernel(const __nv_bfloat16* __restrict__ ym, const int* __restrict__ dst
   }
 }
 
+// LayerNorm over the 1024 channels of every row (the pre-norm of the transformer blocks, Sec. 3.1):
+// y = (x - mean) / sqrt(var + eps) * gamma + beta, population variance, two passes over the row held
+// in registers, fp32, one rounding.  One warp per row like the kernels above.
+__global__ void __launch_bounds__(kRowThreads)
+layernorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
+                 const __nv_bfloat16* __restrict__ beta, __nv_bfloat16* __restrict__ out, long long rows, float eps) {
+  const int lane = threadIdx.x & 31;
+  const long long i = (long long)blockIdx.x * kRowsPerCta + (threadIdx.x >> 5);
+  if (i >= rows) return;
+  uint4 v[4];
+  load_row(v, x + i * 1024, lane);
+  float f[32];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      f[q * 8 + 2 * k] = bf16_lo(w[k]);
+      f[q * 8 + 2 * k + 1] = bf16_hi(w[k]);
+    }
+  }
+  float sum = 0.0f;
+#pragma unroll
+  for (int k = 0; k < 32; ++k) sum += f[k];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum * (1.0f / 1024.0f);
+  float ss = 0.0f;
+#pragma unroll
+  for (int k = 0; k < 32; ++k) {
+    f[k] -= mean;
+    ss = fmaf(f[k], f[k], ss);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rstd = rsqrtf(ss * (1.0f / 1024.0f) + eps);
+  uint4* op = reinterpret_cast<uint4*>(out + i * 1024);
+  const uint4* gp = reinterpret_cast<const uint4*>(gamma);
+  const uint4* bp = reinterpret_cast<const uint4*>(beta);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 g = gp[q * 32 + lane], b = bp[q * 32 + lane];
+    const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      c[k] = pack_bf16(fmaf(f[q * 8 + 2 * k] * rstd, bf16_lo(gw[k]), bf16_lo(bw[k])),
+                       fmaf(f[q * 8 + 2 * k + 1] * rstd, bf16_hi(gw[k]), bf16_hi(bw[k])));
+    op[q * 32 + lane] = make_uint4(c[0], c[1], c[2], c[3]);
+  }
+}
+
+cudaError_t launch_layernorm(const __nv_bfloat16* x, const __nv_bfloat16* gamma, const __nv_bfloat16* beta,
+                             __nv_bfloat16* out, long long rows, float eps, cudaStream_t s, int* launches) {
+  if (rows == 0) return cudaSuccess;
+  const unsigned blocks = (unsigned)((rows + kRowsPerCta - 1) / kRowsPerCta);
+  layernorm_kernel<<<blocks, kRowThreads, 0, s>>>(x, gamma, beta, out, rows, eps);
+  ++*launches;
+  return cudaGetLastError();
+}
+
 cudaError_t launch_merge(const litevggt_ctx* ctx, const litevggt_plan* plan, const __nv_bfloat16* x,
                          __nv_bfloat16* xm, cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;

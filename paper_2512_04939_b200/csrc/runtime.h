@@ -25,6 +25,8 @@ struct Sizes {
 
 inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
 
+constexpr long long kMlpChunkRows = 131072;  // rows of the 4D-wide hidden activations held at a time (1 GiB)
+
 // One device allocation carved into named regions.
 struct Workspace {
   uint8_t* base = nullptr;
@@ -56,6 +58,10 @@ struct Workspace {
   __nv_bfloat16* stage_xm = nullptr;  // [M, D]
   __nv_bfloat16* stage_ym = nullptr;  // [M, D]
   __nv_bfloat16* stage_out = nullptr; // [N, D]
+  // block workspace of the frame-local attention and the MLP (allocated on first use)
+  __nv_bfloat16* blk_qkv = nullptr;   // [N, 3D]
+  __nv_bfloat16* blk_o = nullptr;     // [N, D]
+  __nv_bfloat16* blk_hidden = nullptr; // [kMlpChunkRows, 4D]
   uint32_t* status = nullptr;         // device status word
 };
 
@@ -64,7 +70,7 @@ struct Workspace {
 namespace lv {
 // Device-time stopwatches, one per step of the path: CUDA event pairs recorded on the
 // launching stream around the step's kernels, kept in a small ring per step.
-constexpr int kNumTimers = 10;
+constexpr int kNumTimers = 13;
 constexpr int kTimerSlots = 64;
 struct Timers {
   cudaEvent_t start[kNumTimers][kTimerSlots];
@@ -149,9 +155,16 @@ cudaError_t launch_unmerge(const litevggt_ctx* ctx, const litevggt_plan* plan, c
 cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k, const __nv_bfloat16* w,
                           long long n, const __nv_bfloat16* bias, __nv_bfloat16* out, cudaStream_t s, int* launches);
 
+cudaError_t launch_linear_mlp(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k,
+                              const __nv_bfloat16* w, long long n, const __nv_bfloat16* bias, int gelu,
+                              const __nv_bfloat16* residual, __nv_bfloat16* out, cudaStream_t s, int* launches);
+cudaError_t launch_layernorm(const __nv_bfloat16* x, const __nv_bfloat16* gamma, const __nv_bfloat16* beta,
+                             __nv_bfloat16* out, long long rows, float eps, cudaStream_t s, int* launches);
+
 // attention.cu
-cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long m, __nv_bfloat16* o,
-                                   cudaStream_t s, int* launches);
+// n_seq independent sequences of seq_len rows each, laid back to back in qkv / o
+cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long seq_len, int n_seq,
+                                   __nv_bfloat16* o, cudaStream_t s, int* launches);
 size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset);
 
 }  // namespace lv

@@ -10,5 +10,6 @@ from .generate import (  # noqa: F401
     make_images,
     make_tokens,
     make_attention_weights,
+    make_block_weights,
     make_workload_inputs,
 )

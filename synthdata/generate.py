@@ -221,6 +221,26 @@ def make_attention_weights(wl: Workload, layer: int, device="cpu", dim: int = DI
     return w_qkv, b_qkv, w_o, b_o
 
 
+def make_block_weights(wl: Workload, layer: int, device="cpu", dim: int = DIM):
+    """Weights of the other sub-layers of one aggregator block, bf16: two LayerNorms (gamma near 1,
+    beta near 0), the frame-attention layer (as make_attention_weights) and the MLP of ratio 4
+    (w1 [4*dim, dim], b1, w2 [dim, 4*dim], b2 ~ N(0, 0.02^2))."""
+    dev = torch.device(device)
+    g = _gen(wl.seed + 500 + layer, dev)
+    bf = torch.bfloat16
+    ln = [((1.0 + 0.1 * torch.randn(dim, generator=g, device=dev)).to(bf), (0.1 * torch.randn(dim, generator=g, device=dev)).to(bf))
+          for _ in range(2)]
+    attn = [(0.02 * torch.randn(3 * dim, dim, generator=g, device=dev)).to(bf),
+            (0.02 * torch.randn(3 * dim, generator=g, device=dev)).to(bf),
+            (0.02 * torch.randn(dim, dim, generator=g, device=dev)).to(bf),
+            (0.02 * torch.randn(dim, generator=g, device=dev)).to(bf)]
+    mlp = [(0.02 * torch.randn(4 * dim, dim, generator=g, device=dev)).to(bf),
+           (0.02 * torch.randn(4 * dim, generator=g, device=dev)).to(bf),
+           (0.02 * torch.randn(dim, 4 * dim, generator=g, device=dev)).to(bf),
+           (0.02 * torch.randn(dim, generator=g, device=dev)).to(bf)]
+    return dict(ln1=ln[0], ln2=ln[1], attn=attn, mlp=mlp)
+
+
 def make_workload_inputs(name: str, device="cpu"):
     """Convenience: (workload, images fp32 [F,3,H,W], tokens bf16 [N,D])."""
     wl = WORKLOADS[name]

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle as O
-from synthdata import WORKLOADS, Workload, make_attention_weights, make_images, make_tokens
+from synthdata import WORKLOADS, Workload, make_attention_weights, make_block_weights, make_images, make_tokens
 from helpers import bf16_bound, rel_err, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -165,6 +165,33 @@ def test_identity_at_ratio_zero_and_reuse_equals_recompute(lib):
     p.destroy(); ctx.close()
 
 
+# ------------------------------------------------------------------ naive (fixed-stride) anchors
+def test_fixed_stride_anchor_rule(lib):
+    """The partition the paper argues against (Sec. 3.2: fixed-stride dst tokens, nothing protected)
+    is the same code path with the GA map switched off: alpha = beta = 0 makes every score tie, ties
+    go to the lowest index, so each 2x2 cell's anchor is its top-left token; ga_keep_frac = 0 leaves
+    no GA tokens."""
+    wl = ODD
+    img, tok = _inputs(wl)
+    grad = O.grad_map(img.numpy())
+    ref = O.merge_plan(to_f64(tok), grad, wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio,
+                       ga_keep_frac=0.0, alpha=0.0, beta=0.0)
+    ctx = lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, ga_keep_frac=0.0, alpha=0.0, beta=0.0)
+    assert (ctx.n_src, ctx.n_dst, ctx.n_merged) == (ref["sizes"]["n_src"], ref["sizes"]["n_dst"], ref["sizes"]["M"])
+    plan = ctx.merge_plan(tok.cuda(), torch.from_numpy(grad.astype(np.float32)).cuda())
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    assert np.array_equal(ex["cls"], ref["cls"])
+    per_frame = ex["cls"].reshape(wl.frames, wl.tokens_per_frame)[1:, 5:].reshape(-1, wl.grid_h, wl.grid_w)
+    assert not np.any(per_frame == O.CLS_GA)
+    assert np.all(per_frame[:, ::2, ::2] == O.CLS_DST) and (per_frame == O.CLS_DST).sum() == (wl.frames - 1) * 5 * 6
+    _check_match(ex, ref)
+    dst_of, size, kept = O.select_and_index(ref["cls"], ex["best_dst"], ex["best_sim"], ref["sizes"]["R"])
+    assert np.array_equal(ex["dst_of"], dst_of) and np.array_equal(ex["size"], size)
+    plan.destroy()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ a6 / a10 merge, unmerge
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
 def test_merge_unmerge_with_oracle_plan(lib, wl):
@@ -258,6 +285,46 @@ def test_global_attention(lib, wl):
             # three stored bf16 intermediates (qkv, o, y) instead of one rounding: the floor of
             # the chain is about twice that of a single rounding at the 4-5 sigma entries
             assert rel_err(to_f64(y), ref_full) <= 2 * bf16_bound(ref_full), "attention layer end to end"
+    ctx.close()
+
+
+# ------------------------------------------------------------------ other sub-layers of a block
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD], ids=lambda w: w.name)
+def test_layernorm_frame_attention_and_mlp(lib, wl):
+    _, tok = _inputs(wl)
+    w = make_block_weights(wl, 0)
+    ctx = _ctx(lib, wl)
+    x = tok.cuda()
+    x64 = to_f64(tok)
+    # LayerNorm: fp32 two-pass statistics, one rounding
+    g, b = w["ln1"]
+    xn = ctx.layernorm(x, g.cuda(), b.cuda(), eps=1e-6)
+    ctx.poll()
+    ref_n = O.layernorm(x64, to_f64(g), to_f64(b), 1e-6)
+    assert rel_err(to_f64(xn), ref_n) <= bf16_bound(ref_n)
+    # frame-local attention on the GPU's own normalised rows, residual = the block input
+    aw = [t.cuda() for t in w["attn"]]
+    y = ctx.frame_attn(xn, *aw, residual=x)
+    ctx.poll()
+    ref_y = O.frame_attention(to_f64(xn), wl.frames, *[to_f64(t) for t in w["attn"]], heads=16, residual=x64)
+    # qkv, o and y are stored in bf16 on the way: twice the single-rounding bound, as for the
+    # global layer end to end
+    assert rel_err(to_f64(y), ref_y) <= 2 * bf16_bound(ref_y)
+    # no token may see another frame: perturbing one frame must leave the others' rows bit-identical
+    x2 = xn.clone()
+    t = wl.tokens_per_frame
+    x2[t:2 * t] += 1.0
+    y2 = ctx.frame_attn(x2, *aw, residual=x)
+    ctx.poll()
+    keep = torch.ones(wl.n_tokens, dtype=torch.bool, device="cuda")
+    keep[t:2 * t] = False
+    assert torch.equal(y[keep], y2[keep]) and not torch.equal(y[~keep], y2[~keep])
+    # MLP with exact GELU; the hidden activations are stored in bf16
+    mw = [t_.cuda() for t_ in w["mlp"]]
+    z = ctx.mlp(xn, *mw, residual=x)
+    ctx.poll()
+    ref_z = O.mlp(to_f64(xn), *[to_f64(t_) for t_ in w["mlp"]], residual=x64)
+    assert rel_err(to_f64(z), ref_z) <= 2 * bf16_bound(ref_z)
     ctx.close()
 
 

@@ -437,3 +437,63 @@ def test_cached_plan_equals_recomputed_plan_on_unchanged_features():
     x_new = x + 0.1 * RNG.standard_normal(x.shape)
     xm = O.merge(x_new, a["dst_of"], a["sizes"]["M"])
     np.testing.assert_allclose((a["size"][:, None] * xm).sum(0), x_new.sum(0), rtol=1e-11)
+
+
+def test_partition_without_scores_is_the_fixed_stride_rule():
+    # alpha = beta = 0: every GA score ties, ties go to the lowest index, so each 2x2 cell's anchor is
+    # its top-left token; with no GA tokens kept this is the fixed-stride partition of Sec. 3.2
+    ga = O.ga_map(RNG.random((3, 9, 11)), RNG.random((3, 9, 11)), alpha=0.0, beta=0.0)
+    assert np.all(ga == 0.0)
+    cls = O.partition(ga, ga_keep_frac=0.0).reshape(3, -1)
+    assert np.all(cls[0, 5:] == O.CLS_DST)
+    grid = cls[1:, 5:].reshape(-1, 9, 11)
+    expect = np.full((9, 11), O.CLS_SRC)
+    expect[::2, ::2] = O.CLS_DST
+    assert np.all(grid == expect)
+    s = O.derived_sizes(3, 9, 11, ga_keep_frac=0.0)
+    assert (s["n_dst_frame"], s["n_ga_frame"], s["n_src_frame"]) == (30, 0, 69)
+
+
+# ------------------------------------------------------------------ other sub-layers of a block
+def test_layernorm_against_library_routine_and_invariants():
+    x = RNG.normal(size=(7, 1024)) * 3.0 + 1.5
+    g, b = RNG.normal(size=1024), RNG.normal(size=1024)
+    ref = F.layer_norm(torch.from_numpy(x), (1024,), torch.from_numpy(g), torch.from_numpy(b), eps=1e-6).numpy()
+    np.testing.assert_allclose(O.layernorm(x, g, b, 1e-6), ref, atol=1e-12)
+    y = O.layernorm(x, np.ones(1024), np.zeros(1024), 1e-12)
+    np.testing.assert_allclose(y.mean(1), 0.0, atol=1e-12)
+    np.testing.assert_allclose((y * y).mean(1), 1.0, atol=1e-9)
+    # invariant to shifting and positive scaling of a row (up to eps)
+    np.testing.assert_allclose(O.layernorm(5.0 * x + 2.0, g, b, 1e-12), O.layernorm(x, g, b, 1e-12), atol=1e-9)
+
+
+def test_gelu_and_mlp_against_library_routine():
+    x = RNG.normal(size=(5, 64)) * 2.0
+    np.testing.assert_allclose(O.gelu(x), F.gelu(torch.from_numpy(x)).numpy(), atol=1e-14)
+    assert O.gelu(np.zeros(3)).tolist() == [0.0, 0.0, 0.0]
+    assert O.gelu(np.array([10.0]))[0] == pytest.approx(10.0, rel=1e-12) and abs(O.gelu(np.array([-10.0]))[0]) < 1e-20
+    w1, b1 = RNG.normal(size=(256, 64)), RNG.normal(size=256)
+    w2, b2 = RNG.normal(size=(64, 256)), RNG.normal(size=64)
+    t = lambda a: torch.from_numpy(a)
+    ref = F.linear(F.gelu(F.linear(t(x), t(w1), t(b1))), t(w2), t(b2)) + t(x)
+    np.testing.assert_allclose(O.mlp(x, w1, b1, w2, b2, residual=x), ref.numpy(), atol=1e-10)
+
+
+def test_frame_attention_is_global_attention_under_a_block_diagonal_mask():
+    frames, t, d, heads = 3, 7, 32, 2
+    x = RNG.normal(size=(frames * t, d))
+    w_qkv, b_qkv = RNG.normal(size=(3 * d, d)) * 0.3, RNG.normal(size=3 * d) * 0.1
+    w_o, b_o = RNG.normal(size=(d, d)) * 0.3, RNG.normal(size=d) * 0.1
+    got = O.frame_attention(x, frames, w_qkv, b_qkv, w_o, b_o, heads=heads, residual=x)
+    # brute force: full attention with scores between different frames set to -inf
+    qkv = x @ w_qkv.T + b_qkv
+    dh = d // heads
+    o = np.zeros_like(x)
+    frame_of = np.repeat(np.arange(frames), t)
+    for h in range(heads):
+        q, k, v = (qkv[:, i * d + h * dh:i * d + (h + 1) * dh] for i in range(3))
+        s = q @ k.T / math.sqrt(dh)
+        s[frame_of[:, None] != frame_of[None, :]] = -np.inf
+        p = np.exp(s - s.max(1, keepdims=True))
+        o[:, h * dh:(h + 1) * dh] = (p / p.sum(1, keepdims=True)) @ v
+    np.testing.assert_allclose(got, o @ w_o.T + b_o + x, atol=1e-12)
