@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
+from synthdata import WORKLOADS, make_attention_weights, make_block_weights, make_images, make_tokens
 
 import hashlib
 
@@ -332,6 +332,51 @@ def run_ours(args, wl):
     ctx.poll()
     e2e_value = aggregate_frames_per_s(wl.frames, args.steps, world, e2e_ms)
 
+    block = None
+    if args.block:
+        # One aggregator block (Sec. 3.1), pre-norm: x += frame_attn(LN x); x += MLP(LN x);
+        # x += unmerge(global_attn(merge(LN x))); x += MLP(LN x).  Plan refreshed every k-th block.
+        bw = make_block_weights(wl, 0, dev)
+        bw2 = make_block_weights(wl, 1, dev)
+        xn = torch.empty(n, d, dtype=torch.bfloat16, device=dev)
+        cur, nxt = bufs[0], bufs[1]
+        cur.copy_(tokens)
+        bstate = {"plan": state["plan"]}
+
+        def run_blocks(count):
+            a, b_ = cur, nxt
+            for idx in range(count):
+                ctx.layernorm(a, *bw["ln1"], out=xn)
+                ctx.frame_attn(xn, *bw["attn"], residual=a, out=b_)
+                ctx.layernorm(b_, *bw["ln2"], out=xn)
+                ctx.mlp(xn, *bw["mlp"], residual=b_, out=a)
+                ctx.layernorm(a, *bw2["ln1"], out=xn)
+                if idx % wl.recompute_interval == 0:
+                    bstate["plan"] = ctx.merge_plan(xn, state["grad"], bstate["plan"])
+                ctx.merge(bstate["plan"], xn, xm)
+                ctx.global_attn(xm, *weights[idx % len(weights)], out=ym)
+                ctx.unmerge(bstate["plan"], ym, a, out=b_)
+                ctx.layernorm(b_, *bw2["ln2"], out=xn)
+                ctx.mlp(xn, *bw2["mlp"], residual=b_, out=a)
+
+        run_blocks(1)
+        ctx.poll()
+        barrier()
+        ctx.timers_reset()
+        ev0.record()
+        run_blocks(args.steps)
+        ev1.record()
+        barrier()
+        blk_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+        ctx.poll()
+        bt = ctx.timers_read()
+        per = lambda k: round(bt[k][0] / max(bt[k][1], 1), 3)
+        block = {"ms_per_block": blk_ms / args.steps, "frames_per_s": aggregate_frames_per_s(wl.frames, args.steps, world, blk_ms),
+                 "ms": {"layernorm (x4)": per("layernorm"), "frame_attn": per("frame_attn"), "mlp (x2)": per("mlp"),
+                        "merge": per("merge"), "global attention core": per("attention"), "unmerge": per("unmerge")},
+                 "note": "one block = frame-local attention + MLP + merged global attention + MLP, pre-norm; "
+                         "plan refreshed every %d blocks" % wl.recompute_interval}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -389,6 +434,8 @@ def run_ours(args, wl):
         "breakdown": breakdown,
         "cpu_baseline": cpu,
     }
+    if block is not None:
+        line["aggregator_block"] = block
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -402,6 +449,9 @@ def main():
     ap.add_argument("--workload", default="C5", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--block", action="store_true",
+                    help="also time whole aggregator blocks (LayerNorm, frame-local attention, MLP around the "
+                         "merged global layer) and add an \"aggregator_block\" object to the line")
     ap.add_argument("--interval", type=int, default=None,
                     help="recompute the merge plan every this many layers (default: the workload's, 6); "
                          "with --steps 24 this reproduces the paper's recompute-interval ablation")

@@ -8,7 +8,7 @@ import pytest
 import torch
 
 import oracle as O
-from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
+from synthdata import WORKLOADS, make_attention_weights, make_block_weights, make_images, make_tokens
 from helpers import bf16_bound, rel_err, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -178,3 +178,27 @@ def test_attention_layer_on_sampled_rows(run):
         half_ulp = float((2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref_o), 1e-30))) - 8)).max()) / rms
         bound = max(1e-2, half_ulp + 2e-3) + 2.0 ** -8 * float(weighted_abs.max()) / rms
         assert rel_err(o_rows[:, 64 * head:64 * head + 64], ref_o) <= bound, f"attention core, head {head}"
+
+
+def test_block_sublayers_on_sampled_rows_and_frames(run):
+    """LayerNorm, frame-local attention and the MLP at N = 1,041,000 rows: sampled rows / whole sampled
+    frames against the oracle, each fed the GPU's own upstream result."""
+    ctx, wl, tokens = run["ctx"], run["wl"], run["tokens"]
+    w = make_block_weights(wl, 0, "cuda")
+    rng = np.random.default_rng(8)
+    rows = np.unique(np.concatenate([rng.choice(wl.n_tokens, 96, replace=False), [0, wl.n_tokens - 1]]))
+    rows_t = torch.from_numpy(rows).cuda()
+    xn = ctx.layernorm(tokens, *w["ln1"], eps=1e-6)
+    ref_n = O.layernorm(to_f64(tokens[rows_t]), to_f64(w["ln1"][0]), to_f64(w["ln1"][1]), 1e-6)
+    assert rel_err(to_f64(xn[rows_t]), ref_n) <= bf16_bound(ref_n)
+    y = ctx.frame_attn(xn, *w["attn"], residual=tokens)
+    z = ctx.mlp(xn, *w["mlp"], residual=tokens)
+    ctx.poll()
+    t = wl.tokens_per_frame
+    aw = [to_f64(u) for u in w["attn"]]
+    for f in (0, 512, 999):
+        sl = slice(f * t, (f + 1) * t)
+        ref_y = O.frame_attention(to_f64(xn[sl]), 1, *aw, heads=16, residual=to_f64(tokens[sl]))
+        assert rel_err(to_f64(y[sl]), ref_y) <= 2 * bf16_bound(ref_y), f"frame attention, frame {f}"
+    ref_z = O.mlp(to_f64(xn[rows_t]), *[to_f64(u) for u in w["mlp"]], residual=to_f64(tokens[rows_t]))
+    assert rel_err(to_f64(z[rows_t]), ref_z) <= 2 * bf16_bound(ref_z)
