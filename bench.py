@@ -40,7 +40,7 @@ METRIC = "frames/s through merge+global-attn+unmerge (plan refreshed every 6th l
 # workload C5, summed over the layer's key-chunk launches, from one single-pass ncu capture
 # (profiles/flash_attention_C5_dram.md).  Reported only while the kernel source is the one that was
 # measured.
-ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 20.24e9 + 8.21e9, "kernel_sha256": "aebbf49d8b710d85ba540fd6c0553fefcfc30eda9f410f03a0e5dcd1d81e7b1d"}
+ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 20.72e9 + 8.21e9, "kernel_sha256": "9c378cfc9d2bf3ce39d0111d70999b197e1bc35bc5b7c67f08795e3d6b644147"}
 
 
 def _attention_source_hash() -> str:

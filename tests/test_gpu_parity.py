@@ -388,6 +388,14 @@ def test_abi_misuse_returns_error_codes(lib):
     with pytest.raises(lib.LiteVGGTError) as e:
         ctx.plan_import(bad)
     assert e.value.code == 3
+    # the block sub-layers validate their arguments too
+    rc = ctx.lib.litevggt_layernorm(ctx.handle, x.data_ptr(), 16, x.data_ptr(), x.data_ptr(), 0.0, x.data_ptr(), None)
+    assert rc == 3  # eps must be positive
+    rc = ctx.lib.litevggt_mlp(ctx.handle, x.data_ptr(), ctx.n_tokens + 1, x.data_ptr(), None, x.data_ptr(), None, None,
+                              x.data_ptr(), None)
+    assert rc == 3  # more rows than the context was sized for
+    rc = ctx.lib.litevggt_frame_attn(ctx.handle, x.data_ptr(), None, None, x.data_ptr(), None, None, x.data_ptr(), None)
+    assert rc == 1  # missing weights
     # a caller partition with wrong class counts is flagged, not followed out of bounds
     cls_bad = torch.from_numpy(ref["cls"].copy())
     cls_bad[wl.tokens_per_frame + 7] = O.CLS_PROTECTED if cls_bad[wl.tokens_per_frame + 7] != O.CLS_PROTECTED else O.CLS_SRC
