@@ -11,16 +11,18 @@
 //               partial row maxima through shared memory once per step.  Four softmax warps
 //               per scheduler keep the special-function unit busy while others wait.
 //   warp  16    MMA issuer of tile 0 (one elected lane):  S_h = Q K_jh^T  and  O += P_h V_jh
-//   warp  17    TMA producer (one elected lane): K_j / V_j through two shared-memory rings
+//   warp  17    TMA producer (one elected lane): K_j / V_j through two 4-stage shared-memory rings
 //   warp  18    MMA issuer of tile 1 (issuing costs tens of cycles per instruction, so one
 //               thread cannot feed both tiles)
 //   warp  19    idle
-// Tensor memory (512 columns allocated, 448 used):
+// Tensor memory (512 columns allocated, 480 used):
 //   [0,256)    S/P: tile t, half h at column t*128 + h*64.  S_th is 128 x 64 fp32; after the
 //              softmax threads have read it they overwrite its first 32 columns with P_th
 //              (bf16 pairs), which the second MMA reads as its A operand from there.
-//   [256,384)  O_0, O_1 (fp32, 64 columns each)
-//   [384,448)  Q_0, Q_1 (bf16 pairs, 32 columns each), written once by the softmax threads
+//   [256,416)  O_0, O_1 (fp32, 80 columns each: 64 output channels, then the row sum - the second
+//              MMA's B operand carries a column of ones next to V, so the tensor core adds up
+//              exactly the bf16 probabilities that it multiplies with V - and 15 unused columns)
+//   [416,480)  Q_0, Q_1 (bf16 pairs, 32 columns each), written once by the softmax threads
 //              straight from global memory: Q is the A operand of the first MMA from tensor
 //              memory, so only K and V tiles travel through shared memory.
 // The two halves of a tile double-buffer the scores: while the softmax threads work on
@@ -55,11 +57,12 @@
 
 namespace lv {
 
-constexpr int kFaStages = 5;
+constexpr int kFaStages = 4;
 constexpr int kFaSoftmaxWarps = 16;
 constexpr int kFaThreads = (kFaSoftmaxWarps + 4) * 32;
 constexpr int kFaTileBytes = 128 * 64 * 2;
-constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 384;
+constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 416;
+constexpr uint32_t kFaOCols = 80;  // 64 output channels, the row sum, 15 unused columns
 constexpr float kFaRescaleThreshold = 8.0f;
 #ifndef LV_FA_CHUNK_TILES
 #define LV_FA_CHUNK_TILES 1024
@@ -83,9 +86,8 @@ struct FaBarriers {
 // partial row maxima swapped between the two threads of a row: [step parity][tile][column half][row]
 struct FaExchange {
   float row_max[2][2][2][128];
-  float row_sum[2][2][128];  // [tile][column half][row], once at the end
 };
-constexpr int kFaSmemBytes = 2 * kFaStages * kFaTileBytes + (int)sizeof(FaExchange) + 512 + 1024;
+constexpr int kFaSmemBytes = 3 * kFaStages * kFaTileBytes + (int)sizeof(FaExchange) + 512 + 1024;
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -128,10 +130,10 @@ __device__ __forceinline__ void drain_ring(uint64_t* full, uint32_t issued, uint
   }
 }
 
-// Exponentials of 32 scores of a row: p = 2^(s * scale - m_ref), packed to bf16 pairs; the fp32
-// values are added to the row's packed partial sums.
+// Exponentials of 32 scores of a row: p = 2^(s * scale - m_ref), packed to bf16 pairs (the row sum
+// is formed by the tensor core from these rounded values).
 __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 scale2, float2 neg_m2,
-                                              float2 (&sum2)[4], uint32_t (&packed)[16]) {
+                                              uint32_t (&packed)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg_m2);
@@ -142,7 +144,6 @@ __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 sc
       p.x = fast_exp2(x.x);
       p.y = fast_exp2(x.y);
     }
-    sum2[i & 3] = __fadd2_rn(sum2[i & 3], p);
     packed[i] = pack_bf16(p.x, p.y);
   }
 }
@@ -161,7 +162,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_k = smem;
   uint8_t* smem_v = smem_k + kFaStages * kFaTileBytes;
-  FaExchange* xchg = reinterpret_cast<FaExchange*>(smem_v + kFaStages * kFaTileBytes);
+  uint8_t* smem_ones = smem_v + kFaStages * kFaTileBytes;  // mirrors the V ring, see below
+  FaExchange* xchg = reinterpret_cast<FaExchange*>(smem_ones + kFaStages * kFaTileBytes);
   FaBarriers* bars = reinterpret_cast<FaBarriers*>(xchg + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -199,6 +201,17 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     mbar_fence_init();
     tma_prefetch_desc(&tmap_qkv);
   }
+  // The row sums come out of the second MMA: its B operand is 80 columns wide, V's 64 channels and,
+  // one descriptor stride (the size of the V ring) further on, a block whose first column is 1 and
+  // whose other columns are 0, so accumulator column 64 collects sum_k P[row, k] of exactly the bf16
+  // probabilities that multiply V.  The block is laid out like a V tile (128-byte rows, 16-byte
+  // chunks XOR-swizzled with the row index modulo 8) and repeated for every ring position.
+  for (int i = threadIdx.x; i < kFaStages * kFaTileBytes / 16; i += kFaThreads) {
+    const int r = i >> 3, chunk = i & 7;  // 128-byte row, 16-byte chunk within it
+    const uint32_t first = chunk == (r & 7) ? 0x00003f80u : 0u;  // bf16 1.0 in logical column 0
+    reinterpret_cast<uint4*>(smem_ones)[i] = make_uint4(first, 0u, 0u, 0u);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes, read by the MMA
   if (warp == 16) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
@@ -236,9 +249,9 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     if (elect_one()) {
       const int t = warp == 16 ? 0 : 1;
       constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64, false, false);
-      constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 64, false, true);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(128, kFaOCols, false, true);
       const uint32_t s_col = tmem_base + kFaColS + t * 128;
-      const uint32_t o_col = tmem_base + kFaColO + t * 64;
+      const uint32_t o_col = tmem_base + kFaColO + t * kFaOCols;
       const uint32_t q_col = tmem_base + kFaColQ + t * 32;
       // S_h = Q (tensor memory) x K[64h .. 64h+63]^T (shared memory, K-major); 4 steps of 16 channels
       auto issue_qk = [&](int h, int stage) {
@@ -269,7 +282,9 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           tc_fence_after();
           // 64 keys of V_j (64 rows of 128 bytes = 8192 bytes per half), 16 keys per instruction:
           // 8 TMEM columns of P, 2048 bytes of V
-          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192), 1024, 1024);
+          // second 64-column block of B = the ones block, one V ring further on
+          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192),
+                                                  kFaStages * kFaTileBytes, 1024);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             umma_ts(o_col, s_col + h * 64 + k * 8, v_desc + 128 * k, idesc_pv,
@@ -309,7 +324,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     const bool row_live = row_local < seq_len;
     const int row = row_base + row_local;  // global row of qkv / o
     const uint32_t s_addr = tmem_base + lane_base + kFaColS + t * 128;
-    const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * 64 + c * 32;
+    const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + c * 32;
+    const uint32_t l_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + 64;  // row sum column (+15 unused)
     {
       // this thread's half (32 channels) of its query row goes to tensor memory as it is
       uint32_t qreg[16];
@@ -340,6 +356,13 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           for (int i = 0; i < 32; ++i) acc[i] = 0u;
         }
         tmem_st32(o_addr, acc);
+        if (c == 1) {
+          uint32_t sum[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) sum[i] = 0u;
+          if (row_live) sum[0] = __float_as_uint(ml_state[((size_t)row * (dim / 64) + head) * 4 + 1]);
+          tmem_st16(l_addr, sum);
+        }
       }
       tmem_st_wait();
       tc_fence_before();
@@ -348,14 +371,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     }
     const float2 scale2 = make_float2(scale_log2e, scale_log2e);
     float m_ref = -INFINITY;  // reference maximum, in log2 units (score * scale * log2 e)
-    float2 l_sum2[4] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f),
-                        make_float2(0.0f, 0.0f)};
-    // per (row, head): reference maximum and the two column halves' partial row sums
-    if (!first_chunk) {
-      const float* ml_row = ml_state + ((size_t)(row_live ? row : 0) * (dim / 64) + head) * 4;
-      m_ref = ml_row[0];
-      l_sum2[0].x = ml_row[1 + c];
-    }
+    // per (row, head) the previous chunk parked the reference maximum and the row sum
+    if (!first_chunk) m_ref = ml_state[((size_t)(row_live ? row : 0) * (dim / 64) + head) * 4];
     bool ok = true;
     int pair_syncs = 0;  // both warps of a pair must pass the same number of pair barriers
     for (int n = 0; n < n_steps; ++n) {
@@ -403,9 +420,6 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           tc_fence_after();
           const float m_new = grow ? mx_scaled : m_ref;
           const float alpha = fast_exp2(m_ref - m_new);
-          const float2 alpha2 = make_float2(alpha, alpha);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) l_sum2[i] = __fmul2_rn(l_sum2[i], alpha2);
           m_ref = m_new;
           uint32_t acc[32];  // this thread's 32 of the row's 64 output channels
           tmem_ld32(o_addr, acc);
@@ -413,33 +427,35 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
 #pragma unroll
           for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * alpha);
           tmem_st32(o_addr, acc);
+          if (c == 1) {  // and the row sum, which is one more accumulator column
+            uint32_t sum[16];
+            tmem_ld16(l_addr, sum);
+            tmem_ld_wait();
+            sum[0] = __float_as_uint(__uint_as_float(sum[0]) * alpha);
+            tmem_st16(l_addr, sum);
+          }
         }
       }
       const float2 neg_m2 = make_float2(-m_ref, -m_ref);
       uint32_t packed[16];
-      softmax_chunk(s, scale2, neg_m2, l_sum2, packed);
+      softmax_chunk(s, scale2, neg_m2, packed);
       tmem_st16(s_addr + h * 64 + c * 16, packed);  // P_th lies over the first 32 columns of S_th
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
     }
-    // row sums of the two column halves
-    const float l_own = ((l_sum2[0].x + l_sum2[0].y) + (l_sum2[1].x + l_sum2[1].y)) +
-                        ((l_sum2[2].x + l_sum2[2].y) + (l_sum2[3].x + l_sum2[3].y));
-    xchg->row_sum[t][c][row_in_tile] = l_own;
     // a warp that gave up early still meets its partner at every barrier the partner may be in
     for (; pair_syncs < n_steps; ++pair_syncs) pair_barrier(barrier_id);
-    pair_barrier(barrier_id);
-    const float l_total = l_own + xchg->row_sum[t][c ^ 1][row_in_tile];
     if (ok && mbar_wait_warp(&bars->o_done[t], 0, ctl)) {
       tc_fence_after();
-      uint32_t acc[32];
+      uint32_t acc[32], sum[16];
       tmem_ld32(o_addr, acc);
+      tmem_ld16(l_addr, sum);
       tmem_ld_wait();
       if (row_live) {
         if (last_chunk) {
-          const float inv = 1.0f / l_total;
+          const float inv = 1.0f / __uint_as_float(sum[0]);
           uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -456,8 +472,10 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
 #pragma unroll
           for (int i = 0; i < 8; ++i) dst[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
           float* ml_row = ml_state + ((size_t)row * (dim / 64) + head) * 4;
-          if (c == 0) ml_row[0] = m_ref;
-          ml_row[1 + c] = l_own;
+          if (c == 0) {
+            ml_row[0] = m_ref;
+            ml_row[1] = __uint_as_float(sum[0]);
+          }
         }
       }
     }
