@@ -1,8 +1,9 @@
-"""Parity at the full benchmark size (1000 frames, N = 1,041,000 tokens, M = 520,500 merged
-rows), in the launch configuration bench.py times: one pass of the whole path on the GPU,
-then every step checked against the CPU oracle on sampled outputs that the oracle can compute
-one by one (it is fed the GPU's own upstream result, so each step is judged in isolation), plus
-the properties that hold at any size.  Tolerances are those of the small-size parity tests."""
+"""Parity at the large configurations - C3 (200 frames), C4 (500 frames, every src token merged)
+and C5 (1000 frames, N = 1,041,000 tokens, M = 520,500 merged rows, the configuration bench.py
+times): one pass of the whole path on the GPU, then every step checked against the CPU oracle on
+sampled outputs that the oracle can compute one by one (it is fed the GPU's own upstream result,
+so each step is judged in isolation), plus the properties that hold at any size.  Tolerances are
+those of the small-size parity tests."""
 import numpy as np
 import pytest
 import torch
@@ -13,14 +14,11 @@ from helpers import bf16_bound, rel_err, to_f64
 
 pytestmark = pytest.mark.gpu
 
-FRAMES_SAMPLED = (0, 1, 377, 999)
-
-
-@pytest.fixture(scope="module")
-def run():
+@pytest.fixture(scope="module", params=["C3", "C4", "C5"])
+def run(request):
     import paper_2512_04939_b200 as pkg
 
-    wl = WORKLOADS["C5"]
+    wl = WORKLOADS[request.param]
     images = make_images(wl, "cuda")
     tokens = make_tokens(wl, images)
     ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio)
@@ -32,12 +30,15 @@ def run():
     out = ctx.unmerge(plan, ym, tokens)
     gathered = ctx.unmerge(plan, ym)
     ctx.poll()
-    r = dict(wl=wl, ctx=ctx, images=images, tokens=tokens, weights=weights, grad=grad, plan=plan, xm=xm, ym=ym,
+    frames_sampled = (0, 1, (3 * wl.frames) // 8 + 2, wl.frames - 1)
+    r = dict(frames_sampled=frames_sampled, wl=wl, ctx=ctx, images=images, tokens=tokens, weights=weights, grad=grad, plan=plan, xm=xm, ym=ym,
              out=out, gathered=gathered, ex=ctx.plan_export(plan), sizes=O.derived_sizes(
                  wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio))
     yield r
     plan.destroy()
     ctx.close()
+    del r
+    torch.cuda.empty_cache()
 
 
 def test_sizes_and_index_invariants(run):
@@ -60,7 +61,7 @@ def test_grad_var_ga_maps_on_sampled_frames(run):
     wl, ex = run["wl"], run["ex"]
     t = wl.tokens_per_frame
     grad_gpu = to_f64(run["grad"])
-    for f in FRAMES_SAMPLED:
+    for f in run["frames_sampled"]:
         ref_g = O.grad_map(run["images"][f:f + 1].cpu().numpy())[0]
         assert np.abs(grad_gpu[f] - ref_g).max() <= 1e-5 * max(ref_g.max(), 1e-3)
         ref_v = O.var_map(to_f64(run["tokens"][f * t:(f + 1) * t]), 1, wl.grid_h, wl.grid_w)[0]
@@ -83,7 +84,7 @@ def test_partition_counts_everywhere_and_classes_on_sampled_frames(run):
     pad[:, :wl.grid_h, :wl.grid_w] = grid
     cells = pad.reshape(wl.frames - 1, pad.shape[1] // 2, 2, pad.shape[2] // 2, 2).sum(axis=(2, 4))
     assert np.all(cells == 1)
-    for f in FRAMES_SAMPLED[1:]:
+    for f in run["frames_sampled"][1:]:
         # the oracle's partition of the GPU's own GA map: classes may differ only at near-ties
         ga = ex["ga"][f:f + 1].astype(np.float64)
         # (the oracle treats the first frame of its input as the all-anchor frame: put a copy in front)
@@ -196,7 +197,7 @@ def test_block_sublayers_on_sampled_rows_and_frames(run):
     ctx.poll()
     t = wl.tokens_per_frame
     aw = [to_f64(u) for u in w["attn"]]
-    for f in (0, 512, 999):
+    for f in (0, wl.frames // 2 + 12, wl.frames - 1):
         sl = slice(f * t, (f + 1) * t)
         ref_y = O.frame_attention(to_f64(xn[sl]), 1, *aw, heads=16, residual=to_f64(tokens[sl]))
         assert rel_err(to_f64(y[sl]), ref_y) <= 2 * bf16_bound(ref_y), f"frame attention, frame {f}"
