@@ -37,7 +37,11 @@
 // what the tensor cores would need.  A fixed share of the exponentials of every row can be
 // evaluated on the FMA pipes instead: round-to-nearest split x = n + f, |f| <= 1/2, a cubic
 // for 2^f (relative error 7.5e-5, far below the bf16 rounding of P) and n added into the
-// exponent field.
+// exponent field.  The share is a build-time constant and defaults to zero: on this part packed
+// fp32 instructions issue every second clock, so the cubic costs the FMA pipe about what ex2 costs
+// the special-function unit, and every share tried measured slower than none.
+// Shared memory: K ring, V ring, and behind the V ring a block of the same size that holds the
+// ones column of the P V operand for every ring position (see the kernel).
 //
 // Key chunks.  All CTAs of a head stream the same K/V, but they drift apart, so their combined
 // working set is the head's whole K/V; beyond about a quarter of the L2 that no longer stays
@@ -45,7 +49,7 @@
 // keys).  Long sequences are therefore swept in chunks of at most kFaChunkTiles key tiles, one
 // launch per chunk: a chunk's K/V of one head (32 MiB) stays in L2 while all query blocks pass
 // over it.  Between launches the un-normalised fp32 output rows, the reference maximum and the
-// partial row sums are parked in global memory (a few GB of traffic per launch instead).
+// row sum are parked in global memory (a few GB of traffic per launch instead).
 //
 // Online softmax in base 2 with a lazily updated reference maximum: the running output
 // is rescaled only when a row maximum grows by more than 2^8 over the reference (the
