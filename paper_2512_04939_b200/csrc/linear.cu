@@ -1,5 +1,7 @@
 // bf16 linear layer out = a w^T + bias on the tcgen05 GEMM mainloop (the QKV and output
-// projections of the attention block, Sec. 3.1).
+// projections of the attention block, Sec. 3.1).  The output leaves the SM through TMA stores of
+// 32-row x 64-column blocks, so `out` needs a 16-byte aligned base and a row pitch (n) that is a
+// multiple of 8 elements.
 #include "gemm_tc.cuh"
 #include "runtime.h"
 
@@ -8,23 +10,23 @@ namespace lv {
 cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k, const __nv_bfloat16* w,
                           long long n, const __nv_bfloat16* bias, __nv_bfloat16* out, cudaStream_t s, int* launches) {
   if (m == 0) return cudaSuccess;
-  CUtensorMap tmap_a, tmap_b;
+  CUtensorMap tmap_a, tmap_b, tmap_out;
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap_a, a, (uint64_t)k, (uint64_t)m, (uint64_t)k, kGemmBK, kGemmBM) ||
-      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_b, w, (uint64_t)k, (uint64_t)n, (uint64_t)k, kGemmBK, kGemmBN))
+      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_b, w, (uint64_t)k, (uint64_t)n, (uint64_t)k, kGemmBK, kGemmBN) ||
+      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_out, out, (uint64_t)n, (uint64_t)m, (uint64_t)n, kGemmOutChunkCols,
+                         32))
     return cudaErrorInvalidValue;
   LinearEpilogue epi;
-  epi.out = out;
   epi.bias = bias;
   epi.m_rows = (int)m;
   epi.n_cols = (int)n;
-  epi.ld_out = n;
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<LinearEpilogue>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kGemmSmemBytes);
   if (e != cudaSuccess) return e;
-  const int m_blocks = (int)((m + kGemmBM - 1) / kGemmBM);
-  const int grid = m_blocks < ctx->num_sms ? m_blocks : ctx->num_sms;
-  gemm_tc_kernel<LinearEpilogue><<<grid, kGemmThreads, kGemmSmemBytes, s>>>(tmap_a, tmap_b, (int)m, (int)n, (int)k,
-                                                                            epi, ctx->ws.status);
+  const long long tiles = ((m + kGemmBM - 1) / kGemmBM) * ((n + kGemmBN - 1) / kGemmBN);
+  const int grid = tiles < ctx->num_sms ? (int)tiles : ctx->num_sms;
+  gemm_tc_kernel<LinearEpilogue><<<grid, gemm_threads<LinearEpilogue>(), kGemmSmemBytes, s>>>(tmap_a, tmap_b, tmap_out, (int)m, (int)n,
+                                                                            (int)k, epi, ctx->ws.status);
   ++*launches;
   return cudaGetLastError();
 }
@@ -35,25 +37,26 @@ cudaError_t launch_linear_mlp(litevggt_ctx* ctx, const __nv_bfloat16* a, long lo
                               const __nv_bfloat16* w, long long n, const __nv_bfloat16* bias, int gelu,
                               const __nv_bfloat16* residual, __nv_bfloat16* out, cudaStream_t s, int* launches) {
   if (m == 0) return cudaSuccess;
-  CUtensorMap tmap_a, tmap_b;
+  CUtensorMap tmap_a, tmap_b, tmap_out;
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap_a, a, (uint64_t)k, (uint64_t)m, (uint64_t)k, kGemmBK, kGemmBM) ||
-      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_b, w, (uint64_t)k, (uint64_t)n, (uint64_t)k, kGemmBK, kGemmBN))
+      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_b, w, (uint64_t)k, (uint64_t)n, (uint64_t)k, kGemmBK, kGemmBN) ||
+      !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_out, out, (uint64_t)n, (uint64_t)m, (uint64_t)n, kGemmOutChunkCols,
+                         32))
     return cudaErrorInvalidValue;
   MlpEpilogue epi;
-  epi.out = out;
   epi.bias = bias;
   epi.residual = residual;
   epi.m_rows = (int)m;
   epi.n_cols = (int)n;
-  epi.ld_out = n;
+  epi.ld_res = n;
   epi.gelu = gelu;
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MlpEpilogue>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kGemmSmemBytes);
   if (e != cudaSuccess) return e;
-  const int m_blocks = (int)((m + kGemmBM - 1) / kGemmBM);
-  const int grid = m_blocks < ctx->num_sms ? m_blocks : ctx->num_sms;
-  gemm_tc_kernel<MlpEpilogue><<<grid, kGemmThreads, kGemmSmemBytes, s>>>(tmap_a, tmap_b, (int)m, (int)n, (int)k, epi,
-                                                                         ctx->ws.status);
+  const long long tiles = ((m + kGemmBM - 1) / kGemmBM) * ((n + kGemmBN - 1) / kGemmBN);
+  const int grid = tiles < ctx->num_sms ? (int)tiles : ctx->num_sms;
+  gemm_tc_kernel<MlpEpilogue><<<grid, gemm_threads<MlpEpilogue>(), kGemmSmemBytes, s>>>(tmap_a, tmap_b, tmap_out, (int)m, (int)n,
+                                                                         (int)k, epi, ctx->ws.status);
   ++*launches;
   return cudaGetLastError();
 }

@@ -90,7 +90,8 @@ cudaError_t launch_match(litevggt_ctx* ctx, const __nv_bfloat16* x, int* best_ds
   if (e != cudaSuccess) return e;
   const int m_blocks = (int)((z.n_src + kGemmBM - 1) / kGemmBM);
   const int grid = m_blocks < ctx->num_sms ? m_blocks : ctx->num_sms;
-  gemm_tc_kernel<ArgmaxEpilogue><<<grid, kGemmThreads, kGemmSmemBytes, s>>>(tmap_a, tmap_b, (int)z.n_src,
+  // the argmax epilogue writes no matrix: the store map is never read, any valid map fills the slot
+  gemm_tc_kernel<ArgmaxEpilogue><<<grid, gemm_threads<ArgmaxEpilogue>(), kGemmSmemBytes, s>>>(tmap_a, tmap_b, tmap_a, (int)z.n_src,
                                                                             (int)z.n_dst, 1024, epi, ws.status);
   ++*launches;
   return cudaGetLastError();
