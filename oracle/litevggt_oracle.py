@@ -282,15 +282,77 @@ def linear(a, w, b=None):
     return y
 
 
+def token_positions(frames, grid_h, grid_w, n_special=5):
+    """Integer (row, column) position of every token for the rotary embedding.  Reading (the paper
+    prints none; VGGT's aggregator, which Sec. 3.1 keeps, works this way): the special tokens of
+    a frame sit at (0, 0) and the patch at grid row py, column px at (py + 1, px + 1).  [N, 2]."""
+    t = grid_h * grid_w + n_special
+    pos = np.zeros((frames, t, 2), dtype=np.int64)
+    py, px = np.divmod(np.arange(grid_h * grid_w), grid_w)
+    pos[:, n_special:, 0] = py + 1
+    pos[:, n_special:, 1] = px + 1
+    return pos.reshape(frames * t, 2)
+
+
+def qk_norm(v, gamma, beta, eps=1e-5):
+    """LayerNorm over the channels of each head (population variance), the normalisation VGGT's
+    attention applies to queries and keys before the scores.  v [M, heads, dh]; gamma, beta [dh]."""
+    v = np.asarray(v, dtype=np.float64)
+    mu = v.mean(axis=-1, keepdims=True)
+    var = ((v - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (v - mu) / np.sqrt(var + eps) * np.asarray(gamma, dtype=np.float64) + np.asarray(beta, dtype=np.float64)
+
+
+def rope_2d(v, pos, base=100.0):
+    """Two-dimensional rotary position embedding of queries or keys.  v [M, heads, dh], pos [M, 2].
+
+    The head's channels split into two halves of width h = dh/2: the first turns with the row
+    position pos[:, 0], the second with the column position pos[:, 1].  Inside a half, channel i
+    (i < h/2) and channel i + h/2 form a plane that is rotated by the angle position * base^(-2i/h).
+    A rotation by an angle proportional to the position makes <rope(q, p), rope(k, p')> depend on
+    p - p' only."""
+    v = np.asarray(v, dtype=np.float64)
+    pos = np.asarray(pos, dtype=np.float64)
+    dh = v.shape[-1]
+    h = dh // 2
+    assert dh % 4 == 0
+    theta = base ** (-2.0 * np.arange(h // 2) / h)  # [h/2]
+    out = np.empty_like(v)
+    for axis in range(2):
+        ang = pos[:, axis, None] * theta[None, :]      # [M, h/2]
+        c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+        a = v[..., axis * h: axis * h + h // 2]
+        b = v[..., axis * h + h // 2: (axis + 1) * h]
+        out[..., axis * h: axis * h + h // 2] = a * c - b * s
+        out[..., axis * h + h // 2: (axis + 1) * h] = b * c + a * s
+    return out
+
+
 def global_attention(xm, w_qkv, b_qkv, w_o, b_o, heads=16, rows=None, chunk=1024,
-                     return_parts=False):
+                     return_parts=False, ext=None):
     """Standard multi-head self-attention over the whole (merged) sequence (Sec. 3.1:
     the frame-global attention concatenates all tokens for full-sequence attention).
 
     qkv = xm @ w_qkv.T + b_qkv (rows [0,D) of w_qkv produce Q, [D,2D) K, [2D,3D) V),
     o = attention_core(qkv), y = o @ w_o.T + b_o.  No positional terms, no mask.
-    rows (optional) restricts the queries."""
+    rows (optional) restricts the queries.
+
+    ext (optional, a dict) switches on what VGGT's own attention has and the paper does not print:
+    "q_gamma", "q_beta", "k_gamma", "k_beta" (+ "eps"): qk_norm of queries and keys;
+    "pos" (+ "base"): rope_2d of queries and keys with one position per row of xm, applied after
+    the normalisation."""
     qkv = linear(xm, w_qkv, b_qkv)
+    if ext is not None:
+        m, d = qkv.shape[0], qkv.shape[1] // 3
+        q = qkv[:, :d].reshape(m, heads, d // heads)
+        k = qkv[:, d:2 * d].reshape(m, heads, d // heads)
+        if "q_gamma" in ext:
+            q = qk_norm(q, ext["q_gamma"], ext["q_beta"], ext.get("eps", 1e-5))
+            k = qk_norm(k, ext["k_gamma"], ext["k_beta"], ext.get("eps", 1e-5))
+        if "pos" in ext:
+            q = rope_2d(q, ext["pos"], ext.get("base", 100.0))
+            k = rope_2d(k, ext["pos"], ext.get("base", 100.0))
+        qkv = np.concatenate([q.reshape(m, d), k.reshape(m, d), qkv[:, 2 * d:]], axis=1)
     o = attention_core(qkv, heads, rows, chunk)
     y = linear(o, w_o, b_o)
     if return_parts:

@@ -497,3 +497,95 @@ def test_frame_attention_is_global_attention_under_a_block_diagonal_mask():
         p = np.exp(s - s.max(1, keepdims=True))
         o[:, h * dh:(h + 1) * dh] = (p / p.sum(1, keepdims=True)) @ v
     np.testing.assert_allclose(got, o @ w_o.T + b_o + x, atol=1e-12)
+
+
+# ------------------------------------------------------------------ QK-norm and the 2-D rotary embedding
+def test_qk_norm_against_library_routine():
+    v = RNG.normal(0.3, 2.0, (9, 4, 16))
+    g, b = RNG.normal(1.0, 0.2, 16), RNG.normal(0.0, 0.2, 16)
+    ref = F.layer_norm(torch.from_numpy(v), (16,), torch.from_numpy(g), torch.from_numpy(b), eps=1e-5).numpy()
+    np.testing.assert_allclose(O.qk_norm(v, g, b, 1e-5), ref, rtol=1e-12, atol=1e-12)
+    # every head is normalised on its own: changing one head leaves the others alone
+    v2 = v.copy()
+    v2[:, 1] *= 7.0
+    out, out2 = O.qk_norm(v, g, b), O.qk_norm(v2, g, b)
+    np.testing.assert_array_equal(out[:, [0, 2, 3]], out2[:, [0, 2, 3]])
+
+
+def test_token_positions_layout():
+    pos = O.token_positions(2, 3, 4, n_special=5)
+    assert pos.shape == (2 * 17, 2)
+    assert (pos[:5] == 0).all() and (pos[17:22] == 0).all()          # special tokens at the origin
+    assert tuple(pos[5]) == (1, 1) and tuple(pos[5 + 3]) == (1, 4)    # first grid row
+    assert tuple(pos[5 + 4]) == (2, 1) and tuple(pos[16]) == (3, 4)   # row-major grid
+    np.testing.assert_array_equal(pos[:17], pos[17:])                 # the same in every frame
+
+
+def test_rope_2d_is_a_rotation_by_position_times_frequency():
+    # complex form: channel i + j*(h/2) of a half are the real and imaginary parts of z_i, and the
+    # embedding multiplies z_i by exp(i * position * base^(-2i/h)); dh = 8 -> h = 4, two planes per half
+    base = 100.0
+    v = RNG.normal(0, 1, (6, 3, 8))
+    pos = np.array([[0, 0], [1, 0], [0, 1], [2, 5], [7, 3], [28, 37]])
+    out = O.rope_2d(v, pos, base)
+    for axis in range(2):
+        half = v[..., 4 * axis: 4 * axis + 4]
+        z = half[..., :2] + 1j * half[..., 2:]
+        theta = np.array([1.0, base ** -0.5])                          # base^(-2i/h), i = 0, 1
+        zr = z * np.exp(1j * pos[:, axis, None, None] * theta)
+        np.testing.assert_allclose(out[..., 4 * axis: 4 * axis + 2], zr.real, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(out[..., 4 * axis + 2: 4 * axis + 4], zr.imag, rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(out[0], v[0])                        # position (0, 0): identity
+    np.testing.assert_array_equal(out[1, :, 4:], v[1, :, 4:])          # column 0: second half untouched
+    np.testing.assert_array_equal(out[2, :, :4], v[2, :, :4])          # row 0: first half untouched
+    np.testing.assert_allclose((out ** 2).sum(-1), (v ** 2).sum(-1), rtol=1e-12)   # norms kept
+
+
+def test_rope_2d_scores_depend_on_relative_position_only():
+    q, k = RNG.normal(0, 1, (1, 2, 64)), RNG.normal(0, 1, (1, 2, 64))
+    def score(pq, pk):
+        a = O.rope_2d(q, np.array([pq]))
+        b = O.rope_2d(k, np.array([pk]))
+        return (a * b).sum(-1)
+    s0 = score((3, 9), (11, 2))
+    np.testing.assert_allclose(score((3 + 6, 9 + 20), (11 + 6, 2 + 20)), s0, rtol=0, atol=1e-11)
+    assert np.abs(score((3, 9), (12, 2)) - s0).max() > 1e-3           # a different offset does change them
+    assert np.abs(score((3, 9), (11, 3)) - s0).max() > 1e-3
+
+
+def test_global_attention_extension_reduces_to_plain_and_to_its_parts():
+    m, d, heads = 40, 32, 2
+    xm = RNG.normal(0, 1, (m, d))
+    wq, bq = RNG.normal(0, 0.2, (3 * d, d)), RNG.normal(0, 0.1, 3 * d)
+    wo, bo = RNG.normal(0, 0.2, (d, d)), RNG.normal(0, 0.1, d)
+    plain = O.global_attention(xm, wq, bq, wo, bo, heads=heads)
+    # all positions at the origin and no normalisation: nothing changes
+    same = O.global_attention(xm, wq, bq, wo, bo, heads=heads, ext={"pos": np.zeros((m, 2))})
+    np.testing.assert_allclose(same, plain, rtol=0, atol=1e-12)
+    # all rows at one common position: scores see only relative positions, so again nothing changes
+    same = O.global_attention(xm, wq, bq, wo, bo, heads=heads, ext={"pos": np.tile([[4, 9]], (m, 1))})
+    np.testing.assert_allclose(same, plain, rtol=0, atol=1e-10)
+    # the full extension against torch: normalise, rotate by hand through the complex form, library attention
+    dh = d // heads
+    g1, b1, g2, b2 = (RNG.normal(1, 0.1, dh), RNG.normal(0, 0.1, dh), RNG.normal(1, 0.1, dh), RNG.normal(0, 0.1, dh))
+    pos = RNG.integers(0, 12, (m, 2))
+    got = O.global_attention(xm, wq, bq, wo, bo, heads=heads,
+                             ext={"q_gamma": g1, "q_beta": b1, "k_gamma": g2, "k_beta": b2, "pos": pos})
+    qkv = torch.from_numpy(xm @ wq.T + bq)
+    q, k, v = [t.reshape(m, heads, dh) for t in qkv.split(d, dim=1)]
+    q = F.layer_norm(q, (dh,), torch.from_numpy(g1), torch.from_numpy(b1), eps=1e-5)
+    k = F.layer_norm(k, (dh,), torch.from_numpy(g2), torch.from_numpy(b2), eps=1e-5)
+    def rot(t):
+        t = t.numpy()
+        h = dh // 2
+        out = np.empty_like(t)
+        theta = 100.0 ** (-2.0 * np.arange(h // 2) / h)
+        for axis in range(2):
+            z = t[..., axis * h: axis * h + h // 2] + 1j * t[..., axis * h + h // 2: (axis + 1) * h]
+            z = z * np.exp(1j * pos[:, axis, None, None] * theta)
+            out[..., axis * h: axis * h + h // 2] = z.real
+            out[..., axis * h + h // 2: (axis + 1) * h] = z.imag
+        return torch.from_numpy(out)
+    o = F.scaled_dot_product_attention(rot(q).transpose(0, 1), rot(k).transpose(0, 1), v.transpose(0, 1))
+    ref = o.transpose(0, 1).reshape(m, d).numpy() @ wo.T + bo
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-10)
