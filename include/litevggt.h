@@ -130,6 +130,36 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
                                      const void* w_qkv, const void* b_qkv, const void* w_o,
                                      const void* b_o, void* y_merged, void* stream);
 
+/* Options of litevggt_global_attn_ext.  The paper prints neither; VGGT's attention layer, which
+ * the method keeps (Sec. 3.1), normalises queries and keys per head and rotates them by their 2-D
+ * position, so weights trained that way need both. */
+typedef struct litevggt_attn_ext {
+  /* Per-head LayerNorm of Q and K over the 64 channels of a head (population variance):
+   * dev bf16 [64] each, 16-byte aligned; all four NULL = no normalisation, otherwise all four. */
+  const void* q_norm_gamma;
+  const void* q_norm_beta;
+  const void* k_norm_gamma;
+  const void* k_norm_beta;
+  float norm_eps;   /* > 0 when the normalisation is on (VGGT: 1e-5) */
+  /* 2-D rotary embedding of Q and K, after the normalisation: non-zero = on.  A head's channels
+   * [0,32) turn with the row position, [32,64) with the column position; inside a half, channel i
+   * (< 16) and channel i+16 form a plane rotated by position * rope_base^(-i/16).  Row r of the
+   * merged sequence has the position of the token that owns it (the plan's kept token): special
+   * tokens (0,0), the patch at grid row py, column px (py+1, px+1). */
+  int32_t rope;
+  float rope_base;  /* > 1 when the rotation is on (VGGT: 100) */
+} litevggt_attn_ext;
+
+/* litevggt_global_attn with the options above applied to the projected Q and K before the scores
+ * (normalisation first, then rotation), fp32 arithmetic, one rounding back to bf16.  plan: the plan
+ * the merged rows came from (read for the rows' positions; may be NULL when ext->rope == 0).
+ * Everything else as in litevggt_global_attn.  A LayerScale factor on the layer's output needs no
+ * option: scale the rows of w_o and the entries of b_o by it. */
+litevggt_status litevggt_global_attn_ext(litevggt_ctx* ctx, const litevggt_plan* plan,
+                                         const void* x_merged, int64_t m, const void* w_qkv,
+                                         const void* b_qkv, const void* w_o, const void* b_o,
+                                         const litevggt_attn_ext* ext, void* y_merged, void* stream);
+
 /* The same attention layer as litevggt_global_attn for callers that must not allocate (the paper
  * has no counterpart; this is a property of the library, not of the method).  It needs no
  * context: a context's workspace comes from cudaMalloc, which is off limits for code running
@@ -229,7 +259,7 @@ litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
  * the launching stream: which = 0 grad map, 1 var map, 2 partition + token lists, 3 cosine
  * matching (pack + GEMM/argmax), 4 selection + index build, 5 merge, 6 qkv projection,
  * 7 attention core, 8 output projection, 9 unmerge, 10 LayerNorm, 11 frame-local attention layer,
- * 12 MLP.  litevggt_timers_reset forgets all
+ * 12 MLP, 13 Q/K normalisation + rotary embedding.  litevggt_timers_reset forgets all
  * records; litevggt_timer_read synchronises on the recorded events and returns the summed
  * device time (ms) and the number of records (at most 64 are kept per step). */
 litevggt_status litevggt_timers_reset(litevggt_ctx* ctx);

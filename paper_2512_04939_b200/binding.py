@@ -39,6 +39,12 @@ def library_path() -> str:
     return os.path.join(_HERE, "liblitevggt.so")
 
 
+class AttnExt(C.Structure):
+    """Mirror of litevggt_attn_ext."""
+    _fields_ = [("q_norm_gamma", C.c_void_p), ("q_norm_beta", C.c_void_p), ("k_norm_gamma", C.c_void_p),
+                ("k_norm_beta", C.c_void_p), ("norm_eps", C.c_float), ("rope", C.c_int32), ("rope_base", C.c_float)]
+
+
 def load_library():
     """Load liblitevggt.so (once).  Raises if it has not been built: there is no fallback."""
     global _LIB
@@ -61,6 +67,7 @@ def load_library():
         "litevggt_merge": [vp, vp, vp, vp, vp],
         "litevggt_global_attn": [vp, vp, i64, vp, vp, vp, vp, vp, vp],
         "litevggt_global_attn_static": [vp, i64, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_global_attn_ext": [vp, vp, vp, i64, vp, vp, vp, vp, P(AttnExt), vp, vp],
         "litevggt_unmerge": [vp, vp, vp, vp, vp, vp],
         "litevggt_layernorm": [vp, vp, i64, vp, vp, C.c_float, vp, vp],
         "litevggt_frame_attn": [vp, vp, vp, vp, vp, vp, vp, vp, vp],
@@ -216,6 +223,26 @@ class LiteVGGT:
                                              _ptr(w_o), _ptr(b_o), _ptr(out), _stream()), "global_attn")
         return out
 
+    def global_attn_ext(self, plan, xm, w_qkv, b_qkv, w_o, b_o, q_norm=None, k_norm=None, norm_eps=1e-5,
+                        rope=False, rope_base=100.0, out: torch.Tensor | None = None) -> torch.Tensor:
+        """global_attn with per-head LayerNorm of Q and K (q_norm, k_norm: (gamma, beta) pairs of bf16 [64]
+        tensors, both or neither) and / or the 2-D rotary embedding (positions come from ``plan``)."""
+        assert xm.dtype == torch.bfloat16 and xm.shape == (self.n_merged, self.dim)
+        if out is None:
+            out = torch.empty_like(xm)
+        ext = AttnExt()
+        qg, qb = q_norm if q_norm is not None else (None, None)
+        kg, kb = k_norm if k_norm is not None else (None, None)
+        ext.q_norm_gamma, ext.q_norm_beta, ext.k_norm_gamma, ext.k_norm_beta = _ptr(qg), _ptr(qb), _ptr(kg), _ptr(kb)
+        ext.norm_eps = norm_eps
+        ext.rope = 1 if rope else 0
+        ext.rope_base = rope_base
+        h = plan.handle if plan is not None else None
+        _check(self.lib.litevggt_global_attn_ext(self.handle, h, _ptr(xm), self.n_merged, _ptr(w_qkv), _ptr(b_qkv),
+                                                 _ptr(w_o), _ptr(b_o), C.byref(ext), _ptr(out), _stream()),
+               "global_attn_ext")
+        return out
+
     def unmerge(self, plan: Plan, ym, residual=None, out: torch.Tensor | None = None) -> torch.Tensor:
         assert ym.dtype == torch.bfloat16 and ym.shape == (self.n_merged, self.dim)
         if out is None:
@@ -307,7 +334,7 @@ class LiteVGGT:
         return torch.as_tensor(view, device=self.device).view(torch.bfloat16).clone()
 
     TIMER_NAMES = ("grad_map", "var_map", "partition", "match", "index_build", "merge", "qkv_proj",
-                   "attention", "out_proj", "unmerge", "layernorm", "frame_attn", "mlp")
+                   "attention", "out_proj", "unmerge", "layernorm", "frame_attn", "mlp", "qk_embed")
 
     def timers_reset(self):
         _check(self.lib.litevggt_timers_reset(self.handle), "timers_reset")

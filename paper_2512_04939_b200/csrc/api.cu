@@ -482,6 +482,59 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
   return cuda_status(e);
 }
 
+litevggt_status litevggt_global_attn_ext(litevggt_ctx* ctx, const litevggt_plan* plan, const void* x_merged, int64_t m,
+                                         const void* w_qkv, const void* b_qkv, const void* w_o, const void* b_o,
+                                         const litevggt_attn_ext* ext, void* y_merged, void* stream) {
+  if (!ctx_ok(ctx) || x_merged == nullptr || w_qkv == nullptr || w_o == nullptr || y_merged == nullptr ||
+      ext == nullptr)
+    return LITEVGGT_ERR_NULL;
+  if (m != ctx->sz.n_merged) return LITEVGGT_ERR_SHAPE;
+  if (!aligned16(x_merged) || !aligned16(w_qkv) || !aligned16(w_o) || !aligned16(y_merged) ||
+      (b_qkv != nullptr && !aligned16(b_qkv)) || (b_o != nullptr && !aligned16(b_o)))
+    return LITEVGGT_ERR_ALIGN;
+  const void* affine[4] = {ext->q_norm_gamma, ext->q_norm_beta, ext->k_norm_gamma, ext->k_norm_beta};
+  int given = 0;
+  for (const void* a : affine) given += a != nullptr;
+  if (given != 0 && given != 4) return LITEVGGT_ERR_NULL;  // the four vectors come together or not at all
+  for (const void* a : affine)
+    if (a != nullptr && !aligned16(a)) return LITEVGGT_ERR_ALIGN;
+  if (given == 4 && !(ext->norm_eps > 0.0f)) return LITEVGGT_ERR_SHAPE;
+  if (ext->rope != 0) {
+    if (!(ext->rope_base > 1.0f)) return LITEVGGT_ERR_SHAPE;
+    if (plan == nullptr) return LITEVGGT_ERR_NULL;
+    if (!plan_ok(plan) || plan->owner != ctx || !plan->built) return LITEVGGT_ERR_STALE_PLAN;
+  }
+  const int d = ctx->sz.dim;
+  cudaStream_t s = (cudaStream_t)stream;
+  int n = 0;
+  cudaError_t e;
+  {
+    StepTimer t(ctx, 6, s);
+    e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d, static_cast<const __nv_bfloat16*>(w_qkv),
+                      3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.qkv, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 13, s);
+    e = launch_qk_embed(ctx, ctx->ws.qkv, ext->rope != 0 ? plan->kept_idx : nullptr, m,
+                        static_cast<const __nv_bfloat16*>(ext->q_norm_gamma),
+                        static_cast<const __nv_bfloat16*>(ext->q_norm_beta),
+                        static_cast<const __nv_bfloat16*>(ext->k_norm_gamma),
+                        static_cast<const __nv_bfloat16*>(ext->k_norm_beta), ext->norm_eps, ext->rope != 0,
+                        ext->rope_base, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 7, s);
+    e = launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
+  }
+  if (e == cudaSuccess) {
+    StepTimer t(ctx, 8, s);
+    e = launch_linear(ctx, ctx->ws.attn_o, m, d, static_cast<const __nv_bfloat16*>(w_o), d,
+                      static_cast<const __nv_bfloat16*>(b_o), static_cast<__nv_bfloat16*>(y_merged), s, &n);
+  }
+  bump(ctx, n);
+  return cuda_status(e);
+}
+
 litevggt_status litevggt_layernorm(litevggt_ctx* ctx, const void* x, int64_t rows, const void* gamma, const void* beta,
                                    float eps, void* out, void* stream) {
   if (!ctx_ok(ctx) || x == nullptr || gamma == nullptr || beta == nullptr || out == nullptr) return LITEVGGT_ERR_NULL;

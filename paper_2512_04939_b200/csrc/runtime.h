@@ -70,7 +70,7 @@ struct Workspace {
 namespace lv {
 // Device-time stopwatches, one per step of the path: CUDA event pairs recorded on the
 // launching stream around the step's kernels, kept in a small ring per step.
-constexpr int kNumTimers = 13;
+constexpr int kNumTimers = 14;
 constexpr int kTimerSlots = 64;
 struct Timers {
   cudaEvent_t start[kNumTimers][kTimerSlots];
@@ -163,6 +163,11 @@ cudaError_t launch_layernorm(const __nv_bfloat16* x, const __nv_bfloat16* gamma,
 
 // attention.cu
 // n_seq independent sequences of seq_len rows each, laid back to back in qkv / o
+// qk_embed.cu: optional per-head LayerNorm and 2-D rotary embedding of Q and K, in place on [m, 3D]
+cudaError_t launch_qk_embed(const litevggt_ctx* ctx, __nv_bfloat16* qkv, const int* kept_idx, long long m,
+                            const __nv_bfloat16* q_gamma, const __nv_bfloat16* q_beta, const __nv_bfloat16* k_gamma,
+                            const __nv_bfloat16* k_beta, float eps, int rope, float rope_base, cudaStream_t s,
+                            int* launches);
 cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long seq_len, int n_seq,
                                    __nv_bfloat16* o, cudaStream_t s, int* launches);
 size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset);

@@ -203,3 +203,32 @@ def test_block_sublayers_on_sampled_rows_and_frames(run):
         assert rel_err(to_f64(y[sl]), ref_y) <= 2 * bf16_bound(ref_y), f"frame attention, frame {f}"
     ref_z = O.mlp(to_f64(xn[rows_t]), *[to_f64(u) for u in w["mlp"]], residual=to_f64(tokens[rows_t]))
     assert rel_err(to_f64(z[rows_t]), ref_z) <= 2 * bf16_bound(ref_z)
+
+
+def test_qk_norm_and_rope_on_sampled_rows(run):
+    """The optional Q/K normalisation and rotary embedding at full size: the transformed Q and K of
+    sampled merged rows (first, last, tile edges, random) against the oracle on those rows, positions
+    taken from the owner tokens.  Runs last in this module: it overwrites the layer's intermediates."""
+    ctx, xm, sz, wl, ex = run["ctx"], run["xm"], run["sizes"], run["wl"], run["ex"]
+    w_qkv, b_qkv, w_o, b_o = run["weights"]
+    gen = torch.Generator().manual_seed(wl.seed + 77)
+    affine = [(1.0 + 0.2 * torch.randn(64, generator=gen)).to(torch.bfloat16) if i % 2 == 0
+              else (0.2 * torch.randn(64, generator=gen)).to(torch.bfloat16) for i in range(4)]
+    dev = [t.cuda() for t in affine]
+    y = ctx.global_attn_ext(run["plan"], xm, w_qkv, b_qkv, w_o, b_o, q_norm=(dev[0], dev[1]), k_norm=(dev[2], dev[3]),
+                            rope=True)
+    ctx.poll()
+    m = sz["M"]
+    rng = np.random.default_rng(13)
+    rows = np.unique(np.concatenate([rng.choice(m, 200, replace=False), [0, 7, 8, 127, 128, m - 8, m - 1]]))
+    rows_t = torch.from_numpy(rows).cuda()
+    ref = O.linear(to_f64(xm[rows_t]), to_f64(w_qkv), to_f64(b_qkv))
+    pos = O.token_positions(wl.frames, wl.grid_h, wl.grid_w)[ex["kept_idx"][rows]]
+    got = to_f64(ctx.debug_buffer(0)[rows_t])
+    for name, c0, g, b in (("Q", 0, affine[0], affine[1]), ("K", 1024, affine[2], affine[3])):
+        part = ref[:, c0:c0 + 1024].reshape(len(rows), 16, 64)
+        part = O.rope_2d(O.qk_norm(part, to_f64(g), to_f64(b), 1e-5), pos, 100.0).reshape(len(rows), 1024)
+        assert rel_err(got[:, c0:c0 + 1024], part) <= 2 * bf16_bound(part), name
+    assert rel_err(got[:, 2048:], ref[:, 2048:]) <= bf16_bound(ref[:, 2048:]), "V is only projected"
+    ref_y = O.linear(to_f64(ctx.debug_buffer(1)[rows_t]), to_f64(w_o), to_f64(b_o))
+    assert rel_err(to_f64(y[rows_t]), ref_y) <= bf16_bound(ref_y), "output projection"

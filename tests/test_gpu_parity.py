@@ -288,6 +288,54 @@ def test_global_attention(lib, wl):
     ctx.close()
 
 
+# ------------------------------------------------------------------ Q/K normalisation and rotary embedding
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD], ids=lambda w: w.name)
+@pytest.mark.parametrize("mode", ["norm", "rope", "both"])
+def test_global_attention_with_qk_norm_and_rope(lib, wl, mode):
+    img, tok = _inputs(wl)
+    ctx = _ctx(lib, wl)
+    x = tok.cuda()
+    plan = ctx.merge_plan(x, ctx.grad_map(img.cuda()))
+    ex = ctx.plan_export(plan)
+    xm = ctx.merge(plan, x)
+    w_qkv, b_qkv, w_o, b_o = make_attention_weights(wl, 0)
+    gen = torch.Generator().manual_seed(wl.seed + 77)
+    affine = [(1.0 + 0.2 * torch.randn(64, generator=gen)).to(torch.bfloat16) if i % 2 == 0
+              else (0.2 * torch.randn(64, generator=gen)).to(torch.bfloat16) for i in range(4)]
+    ext = {}
+    if mode in ("norm", "both"):
+        ext.update(q_gamma=to_f64(affine[0]), q_beta=to_f64(affine[1]), k_gamma=to_f64(affine[2]),
+                   k_beta=to_f64(affine[3]), eps=1e-5)
+    if mode in ("rope", "both"):
+        # a merged row sits where the token that owns it sits
+        ext.update(pos=O.token_positions(wl.frames, wl.grid_h, wl.grid_w)[ex["kept_idx"]], base=100.0)
+    dev = [t.cuda() for t in affine]
+    y = ctx.global_attn_ext(plan, xm, w_qkv.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda(),
+                            q_norm=(dev[0], dev[1]) if "q_gamma" in ext else None,
+                            k_norm=(dev[2], dev[3]) if "q_gamma" in ext else None,
+                            rope="pos" in ext)
+    ctx.poll()
+    xm64 = to_f64(xm)
+    w64 = [to_f64(t) for t in (w_qkv, b_qkv, w_o, b_o)]
+    # the transformed Q and K against the oracle's (two roundings on the GPU side: the projection's
+    # output and the transformed values; V must be untouched)
+    ref_y, ref_qkv, _ = O.global_attention(xm64, *w64, heads=16, return_parts=True, ext=ext)
+    qkv = to_f64(ctx.debug_buffer(0))
+    d = 1024
+    for name, sl in (("Q", slice(0, d)), ("K", slice(d, 2 * d)), ("V", slice(2 * d, 3 * d))):
+        assert rel_err(qkv[:, sl], ref_qkv[:, sl]) <= 2 * bf16_bound(ref_qkv[:, sl]), f"{name} after {mode}"
+    plain = to_f64(ctx.linear(xm, w_qkv.cuda(), b_qkv.cuda()))
+    assert np.array_equal(qkv[:, 2 * d:], plain[:, 2 * d:])
+    # the core on the GPU's own transformed Q/K/V, and the layer end to end
+    ref_o = O.attention_core(qkv, heads=16)
+    assert rel_err(to_f64(ctx.debug_buffer(1)), ref_o) <= attention_core_bound(qkv, ref_o), "attention core"
+    assert rel_err(to_f64(y), ref_y) <= 3 * bf16_bound(ref_y), "layer end to end"
+    # and the options did something: Q is far from the plain projection
+    assert rel_err(qkv[:, :d], plain[:, :d]) > 0.5
+    plan.destroy()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ other sub-layers of a block
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD], ids=lambda w: w.name)
 def test_layernorm_frame_attention_and_mlp(lib, wl):
@@ -396,6 +444,23 @@ def test_abi_misuse_returns_error_codes(lib):
     assert rc == 3  # more rows than the context was sized for
     rc = ctx.lib.litevggt_frame_attn(ctx.handle, x.data_ptr(), None, None, x.data_ptr(), None, None, x.data_ptr(), None)
     assert rc == 1  # missing weights
+    # the extended attention layer: options struct required, the four affine vectors come together,
+    # the rotation needs the plan for its positions
+    import ctypes as C
+    xm_ = torch.zeros(ctx.n_merged, 1024, dtype=torch.bfloat16, device="cuda")
+    wq_ = torch.zeros(3072, 1024, dtype=torch.bfloat16, device="cuda")
+    args = lambda plan_h, ext_ref: (ctx.handle, plan_h, xm_.data_ptr(), ctx.n_merged, wq_.data_ptr(), None,
+                                    wq_.data_ptr(), None, ext_ref, xm_.data_ptr(), None)
+    assert ctx.lib.litevggt_global_attn_ext(*args(None, None)) == 1
+    opt = lib.binding.AttnExt()
+    opt.q_norm_gamma = xm_.data_ptr()
+    opt.norm_eps = 1e-5
+    assert ctx.lib.litevggt_global_attn_ext(*args(None, C.byref(opt))) == 1
+    opt = lib.binding.AttnExt()
+    opt.rope, opt.rope_base = 1, 100.0
+    assert ctx.lib.litevggt_global_attn_ext(*args(None, C.byref(opt))) == 1
+    opt.rope_base = 1.0
+    assert ctx.lib.litevggt_global_attn_ext(*args(plan.handle, C.byref(opt))) == 3
     # a caller partition with wrong class counts is flagged, not followed out of bounds
     cls_bad = torch.from_numpy(ref["cls"].copy())
     cls_bad[wl.tokens_per_frame + 7] = O.CLS_PROTECTED if cls_bad[wl.tokens_per_frame + 7] != O.CLS_PROTECTED else O.CLS_SRC
