@@ -308,19 +308,24 @@ def run_ours(args, wl):
     value = aggregate_frames_per_s(wl.frames, args.steps, world, ms)
 
     # ---- end to end through the host-buffer entry point (same schedule, same weights)
+    # Every step is an independent batch: it uploads its own input from pinned memory and downloads its
+    # own result; the entry point runs the copies on the context's copy streams, so they overlap the
+    # neighbouring steps' kernels.  All of it - every copy included - lies inside the timed region.
     x_host = [torch.empty(n, d, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-    x_host[0].copy_(tokens)
+    out_host = [torch.empty(n, d, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    for buf in x_host:
+        buf.copy_(tokens)
     e2e_plan = {"plan": None}
 
     def run_host_steps(count):
         for idx in range(count):
-            src, dst = x_host[idx & 1], x_host[(idx + 1) & 1]
             grad = state["grad"] if idx % wl.recompute_interval == 0 else None
-            e2e_plan["plan"] = ctx.global_layer_host(e2e_plan["plan"], src, *weights[idx], dst, grad=grad)
+            e2e_plan["plan"] = ctx.global_layer_host_pipelined(e2e_plan["plan"], x_host[idx & 1], *weights[idx],
+                                                               out_host[idx & 1], grad=grad)
+        ctx.host_drain()
         torch.cuda.current_stream().synchronize()
 
-    run_host_steps(1)
-    x_host[0].copy_(tokens)
+    run_host_steps(2)
     barrier()
     t0 = time.perf_counter()
     ev0.record()
@@ -419,7 +424,9 @@ def run_ours(args, wl):
         },
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": n * d * 2, "d2h_bytes_per_step": n * d * 2,
-                "ms_per_step": e2e_ms / args.steps},
+                "ms_per_step": e2e_ms / args.steps,
+                "call": "litevggt_global_layer_host_pipelined + litevggt_host_drain: independent steps, pinned "
+                        "host buffers, copies on their own streams overlapping the neighbouring steps' kernels"},
         "gpu_launches": launches,
         "roofline": {"kernel": "flash_attention_kernel", "bound": "tensor", "achieved": att_tflops,
                      "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",

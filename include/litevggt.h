@@ -222,6 +222,28 @@ litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, litevggt_plan** pl
                                            const void* b_qkv, const void* w_o, const void* b_o,
                                            void* out_host, void* stream);
 
+/* litevggt_global_layer_host for a sequence of independent calls (one batch of frames after the
+ * other, as a server would run them): the host-to-device copy of a call's input and the
+ * device-to-host copy of its output run on two copy streams of the context, with double-buffered
+ * staging, so they overlap the neighbouring calls' kernels instead of adding to them (at 1000
+ * frames the two copies are 2 x 2.13 GB, about 6 % of a layer).  Kernels run on `stream`, in call
+ * order.  Arguments as in litevggt_global_layer_host; both host buffers should be pinned.
+ *   - x_host must stay unchanged, and out_host is NOT complete, until litevggt_host_drain has been
+ *     called on `stream` after this call and that point of the stream has been reached.
+ *   - A call does not wait for the output copies of earlier calls: feeding one call's out_host to
+ *     the next call's x_host needs a drain in between (or the plain entry point, which is ordered).
+ *   - The first call allocates the second pair of staging buffers (2 x N x D bf16) and creates the
+ *     streams and events. */
+litevggt_status litevggt_global_layer_host_pipelined(litevggt_ctx* ctx, litevggt_plan** plan_inout,
+                                                     const float* grad, const void* x_host,
+                                                     const void* w_qkv, const void* b_qkv,
+                                                     const void* w_o, const void* b_o,
+                                                     void* out_host, void* stream);
+
+/* Makes `stream` wait for every output copy started by litevggt_global_layer_host_pipelined so far
+ * (no host synchronisation; a no-op when none was started). */
+litevggt_status litevggt_host_drain(litevggt_ctx* ctx, void* stream);
+
 /* Plain bf16 linear layer on the tensor cores: out[m,n] = a[m,k] w[n,k]^T + bias[n].
  * a: dev bf16 [m,k]; w: dev bf16 [n,k]; bias: dev bf16 [n] or NULL; out: dev bf16 [m,n].
  * k and n must be multiples of 64.  This is the projection step of the attention layer. */

@@ -73,6 +73,8 @@ def load_library():
         "litevggt_frame_attn": [vp, vp, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_mlp": [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp],
         "litevggt_global_layer_host": [vp, P(vp), vp, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_global_layer_host_pipelined": [vp, P(vp), vp, vp, vp, vp, vp, vp, vp, vp],
+        "litevggt_host_drain": [vp, vp],
         "litevggt_timers_reset": [vp],
         "litevggt_timer_read": [vp, C.c_int, P(C.c_float), P(i32)],
         "litevggt_linear": [vp, vp, i64, i64, vp, i64, vp, vp, vp],
@@ -261,6 +263,22 @@ class LiteVGGT:
                                                    _ptr(b_qkv), _ptr(w_o), _ptr(b_o), _ptr(out_host), _stream()),
                "global_layer_host")
         return plan if plan is not None else Plan(self, h)
+
+    def global_layer_host_pipelined(self, plan: Plan | None, x_host, w_qkv, b_qkv, w_o, b_o, out_host,
+                                    grad=None) -> Plan:
+        """global_layer_host for independent calls in a row: the copies run on the context's copy
+        streams and overlap the neighbouring calls' kernels.  ``out_host`` is complete only after
+        ``host_drain()`` and a synchronisation of the current stream."""
+        assert x_host.device.type == "cpu" and out_host.device.type == "cpu"
+        assert x_host.shape == (self.n_tokens, self.dim) and out_host.shape == x_host.shape
+        h = plan.handle if plan is not None else C.c_void_p()
+        _check(self.lib.litevggt_global_layer_host_pipelined(self.handle, C.byref(h), _ptr(grad), _ptr(x_host),
+                                                             _ptr(w_qkv), _ptr(b_qkv), _ptr(w_o), _ptr(b_o),
+                                                             _ptr(out_host), _stream()), "global_layer_host_pipelined")
+        return plan if plan is not None else Plan(self, h)
+
+    def host_drain(self):
+        _check(self.lib.litevggt_host_drain(self.handle, _stream()), "host_drain")
 
     def layernorm(self, x, gamma, beta, eps=1e-6, out=None) -> torch.Tensor:
         assert x.dtype == torch.bfloat16 and x.shape[1] == self.dim

@@ -177,6 +177,45 @@ litevggt_status ensure_staging(litevggt_ctx* ctx) {
   return LITEVGGT_OK;
 }
 
+// Copy streams, events and the second pair of [N, D] staging buffers of the pipelined host entry.
+litevggt_status ensure_host_pipe(litevggt_ctx* ctx) {
+  litevggt_status st = ensure_staging(ctx);
+  if (st != LITEVGGT_OK) return st;
+  HostPipe& hp = ctx->pipe;
+  if (hp.created) return LITEVGGT_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LITEVGGT_ERR_CUDA;
+  const size_t big = (size_t)round_up(ctx->sz.n_tokens * ctx->sz.dim * 2, 256);
+  if (cudaMalloc(&hp.extra, 2 * big) != cudaSuccess) {
+    (void)cudaGetLastError();
+    hp.extra = nullptr;
+    return LITEVGGT_ERR_ALLOC;
+  }
+  cudaError_t e = cudaStreamCreateWithFlags(&hp.copy_in, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&hp.copy_out, cudaStreamNonBlocking);
+  cudaEvent_t* sets[4] = {hp.in_ready, hp.x_free, hp.out_ready, hp.out_free};
+  for (int k = 0; k < 4 && e == cudaSuccess; ++k)
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&sets[k][i], cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    // partial set-up is released at destroy time only if `created`; release it here instead
+    if (hp.copy_in) cudaStreamDestroy(hp.copy_in);
+    if (hp.copy_out) cudaStreamDestroy(hp.copy_out);
+    for (int k = 0; k < 4; ++k)
+      for (int i = 0; i < 2; ++i)
+        if (sets[k][i]) cudaEventDestroy(sets[k][i]);
+    cudaFree(hp.extra);
+    hp = HostPipe();
+    return cuda_status(e);
+  }
+  hp.x[0] = ctx->ws.stage_x;
+  hp.out[0] = ctx->ws.stage_out;
+  hp.x[1] = reinterpret_cast<__nv_bfloat16*>(hp.extra);
+  hp.out[1] = reinterpret_cast<__nv_bfloat16*>(hp.extra + big);
+  ctx->ws.bytes += 2 * big;
+  hp.created = true;
+  return LITEVGGT_OK;
+}
+
 litevggt_status ensure_block_ws(litevggt_ctx* ctx) {
   if (ctx->ws.blk_qkv != nullptr) return LITEVGGT_OK;
   const Sizes& z = ctx->sz;
@@ -342,6 +381,17 @@ litevggt_status litevggt_destroy(litevggt_ctx* ctx) {
         cudaEventDestroy(ctx->timers.start[w][i]);
         cudaEventDestroy(ctx->timers.stop[w][i]);
       }
+  if (ctx->pipe.created) {
+    cudaStreamDestroy(ctx->pipe.copy_in);
+    cudaStreamDestroy(ctx->pipe.copy_out);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(ctx->pipe.in_ready[i]);
+      cudaEventDestroy(ctx->pipe.x_free[i]);
+      cudaEventDestroy(ctx->pipe.out_ready[i]);
+      cudaEventDestroy(ctx->pipe.out_free[i]);
+    }
+    if (ctx->pipe.extra != nullptr) cudaFree(ctx->pipe.extra);
+  }
   if (ctx->ws.stage_x != nullptr) cudaFree(ctx->ws.stage_x);
   if (ctx->ws.blk_qkv != nullptr) cudaFree(ctx->ws.blk_qkv);
   if (ctx->ws.base != nullptr) cudaFree(ctx->ws.base);
@@ -657,6 +707,69 @@ litevggt_status litevggt_global_layer_host(litevggt_ctx* ctx, litevggt_plan** pl
   if (st == LITEVGGT_OK) st = litevggt_unmerge(ctx, plan, ws.stage_ym, ws.stage_x, ws.stage_out, stream);
   if (st != LITEVGGT_OK) return st;
   e = cudaMemcpyAsync(out_host, ws.stage_out, bytes, cudaMemcpyDeviceToHost, s);
+  return cuda_status(e);
+}
+
+litevggt_status litevggt_global_layer_host_pipelined(litevggt_ctx* ctx, litevggt_plan** plan_inout, const float* grad,
+                                                     const void* x_host, const void* w_qkv, const void* b_qkv,
+                                                     const void* w_o, const void* b_o, void* out_host, void* stream) {
+  if (!ctx_ok(ctx) || plan_inout == nullptr || x_host == nullptr || out_host == nullptr) return LITEVGGT_ERR_NULL;
+  if (grad == nullptr) {
+    const litevggt_plan* plan = *plan_inout;
+    if (!plan_ok(plan) || plan->owner != ctx || !plan->built) return LITEVGGT_ERR_STALE_PLAN;
+  }
+  litevggt_status st = ensure_host_pipe(ctx);
+  if (st != LITEVGGT_OK) return st;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LITEVGGT_ERR_CUDA;
+  const Sizes& z = ctx->sz;
+  Workspace& ws = ctx->ws;
+  HostPipe& hp = ctx->pipe;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t bytes = (size_t)z.n_tokens * z.dim * 2;
+  const int slot = (int)(hp.calls & 1ull);
+  // copy-in stream: the buffer is free once the unmerge two calls ago has read its residual from it
+  cudaError_t e = cudaSuccess;
+  if (hp.used[slot]) e = cudaStreamWaitEvent(hp.copy_in, hp.x_free[slot], 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(hp.x[slot], x_host, bytes, cudaMemcpyHostToDevice, hp.copy_in);
+  if (e == cudaSuccess) e = cudaEventRecord(hp.in_ready[slot], hp.copy_in);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(s, hp.in_ready[slot], 0);
+  if (e != cudaSuccess) return cuda_status(e);
+  if (grad != nullptr) {
+    st = litevggt_merge_plan(ctx, hp.x[slot], grad, plan_inout, stream);
+    if (st != LITEVGGT_OK) return st;
+  }
+  const litevggt_plan* plan = *plan_inout;
+  st = litevggt_merge(ctx, plan, hp.x[slot], ws.stage_xm, stream);
+  if (st == LITEVGGT_OK)
+    st = litevggt_global_attn(ctx, ws.stage_xm, z.n_merged, w_qkv, b_qkv, w_o, b_o, ws.stage_ym, stream);
+  if (st != LITEVGGT_OK) return st;
+  // the output buffer is free once the copy-out two calls ago has drained it
+  if (hp.used[slot]) e = cudaStreamWaitEvent(s, hp.out_free[slot], 0);
+  if (e != cudaSuccess) return cuda_status(e);
+  st = litevggt_unmerge(ctx, plan, ws.stage_ym, hp.x[slot], hp.out[slot], stream);
+  if (st != LITEVGGT_OK) return st;
+  e = cudaEventRecord(hp.out_ready[slot], s);
+  if (e == cudaSuccess) e = cudaEventRecord(hp.x_free[slot], s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hp.copy_out, hp.out_ready[slot], 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, hp.out[slot], bytes, cudaMemcpyDeviceToHost, hp.copy_out);
+  if (e == cudaSuccess) e = cudaEventRecord(hp.out_free[slot], hp.copy_out);
+  if (e == cudaSuccess) {
+    hp.used[slot] = true;
+    ++hp.calls;
+  }
+  return cuda_status(e);
+}
+
+litevggt_status litevggt_host_drain(litevggt_ctx* ctx, void* stream) {
+  if (!ctx_ok(ctx)) return LITEVGGT_ERR_NULL;
+  HostPipe& hp = ctx->pipe;
+  if (!hp.created) return LITEVGGT_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LITEVGGT_ERR_CUDA;
+  cudaError_t e = cudaSuccess;
+  for (int slot = 0; slot < 2 && e == cudaSuccess; ++slot)
+    if (hp.used[slot]) e = cudaStreamWaitEvent((cudaStream_t)stream, hp.out_free[slot], 0);
   return cuda_status(e);
 }
 

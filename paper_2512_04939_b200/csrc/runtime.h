@@ -80,6 +80,18 @@ struct Timers {
 };
 }  // namespace lv
 
+// Streams, events and the second pair of staging buffers behind litevggt_global_layer_host_pipelined.
+struct HostPipe {
+  bool created = false;
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t in_ready[2] = {}, x_free[2] = {}, out_ready[2] = {}, out_free[2] = {};
+  bool used[2] = {false, false};
+  unsigned long long calls = 0;
+  __nv_bfloat16* x[2] = {nullptr, nullptr};    // [N, D] each
+  __nv_bfloat16* out[2] = {nullptr, nullptr};  // [N, D] each
+  uint8_t* extra = nullptr;                     // allocation that holds x[1] and out[1]
+};
+
 struct litevggt_ctx {
   uint32_t magic;
   litevggt_config cfg;
@@ -90,6 +102,7 @@ struct litevggt_ctx {
   long long launches;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved at run time
   lv::Timers timers;
+  HostPipe pipe;
 };
 
 struct litevggt_plan {

@@ -412,6 +412,50 @@ def test_whole_layer_c1_and_host_entry(lib):
     ctx.close()
 
 
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
+def test_pipelined_host_entry_equals_the_ordered_one(lib, wl):
+    """Five independent calls in a row through the entry point whose copies run on their own streams:
+    each output must be bit-identical to the ordered entry point's on the same input (the kernels are
+    the same; only the copies moved), with the plan refreshed inside the third call."""
+    img, tok = _inputs(wl)
+    ctx = _ctx(lib, wl)
+    grad = ctx.grad_map(img.cuda())
+    w = [t.cuda() for t in make_attention_weights(wl, 0)]
+    gen = torch.Generator().manual_seed(wl.seed + 5)
+    inputs = [tok.clone().pin_memory()]
+    for _ in range(4):
+        inputs.append((tok.float() + 0.05 * torch.randn(tok.shape, generator=gen)).to(torch.bfloat16).pin_memory())
+    # ordered entry point: one call, one synchronisation at a time
+    expected, plan = [], None
+    for i, xh in enumerate(inputs):
+        oh = torch.empty_like(xh).pin_memory()
+        plan = ctx.global_layer_host(plan, xh, *w, oh, grad=grad if i in (0, 2) else None)
+        ctx.poll()
+        expected.append(oh.clone())
+    plan.destroy()
+    outs = [torch.zeros_like(xh).pin_memory() for xh in inputs]
+    plan = None
+    for i, (xh, oh) in enumerate(zip(inputs, outs)):
+        plan = ctx.global_layer_host_pipelined(plan, xh, *w, oh, grad=grad if i in (0, 2) else None)
+    ctx.host_drain()
+    ctx.poll()
+    for i, (got, ref) in enumerate(zip(outs, expected)):
+        assert torch.equal(got, ref), f"call {i}"
+    # a second round reuses both staging slots
+    for xh, oh in zip(inputs[:3], outs[:3]):
+        oh.zero_()
+        ctx.global_layer_host_pipelined(plan, xh, *w, oh)
+    ctx.host_drain()
+    ctx.poll()
+    for i, xh in enumerate(inputs[:3]):
+        oh = torch.empty_like(xh).pin_memory()
+        ctx.global_layer_host(plan, xh, *w, oh)
+        ctx.poll()
+        assert torch.equal(outs[i], oh), f"second round, call {i}"
+    plan.destroy()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ ABI misuse
 def test_abi_misuse_returns_error_codes(lib):
     wl = WORKLOADS["C1"]
