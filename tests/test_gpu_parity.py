@@ -192,6 +192,40 @@ def test_fixed_stride_anchor_rule(lib):
     ctx.close()
 
 
+def test_seeded_random_anchor_rule(lib):
+    """The other naive partition (Sec. 3.2): one anchor per 2x2 cell drawn at random from a seeded
+    generator, nothing protected.  The classes are made on the host (the oracle's partition fed with
+    random scores) and handed to the library, which matches, selects and merges with them; everything
+    downstream is checked against the oracle on the same classes."""
+    wl = ODD
+    _, tok = _inputs(wl)
+    scores = np.random.default_rng(424242).random((wl.frames, wl.grid_h, wl.grid_w))
+    cls = O.partition(scores, ga_keep_frac=0.0)
+    fixed = O.partition(np.zeros_like(scores), ga_keep_frac=0.0)
+    assert (cls != fixed).any() and not np.any(cls == O.CLS_GA)
+    x64 = to_f64(tok)
+    src_idx, dst_idx = np.flatnonzero(cls == O.CLS_SRC), np.flatnonzero(cls == O.CLS_DST)
+    best_dst, sim1, sim2 = O.match(x64, src_idx, dst_idx)
+    ctx = lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, ga_keep_frac=0.0)
+    assert (ctx.n_src, ctx.n_dst) == (src_idx.size, dst_idx.size)
+    x = tok.cuda()
+    plan = ctx.merge_plan_with_partition(x, torch.from_numpy(cls).cuda())
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    assert np.array_equal(ex["cls"], cls)
+    _check_match(ex, dict(best_dst=best_dst, best_sim=sim1, second_sim=sim2))
+    n_remove = O.derived_sizes(wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio, ga_keep_frac=0.0)["R"]
+    dst_of, size, kept = O.select_and_index(cls, ex["best_dst"], ex["best_sim"], n_remove)
+    assert np.array_equal(ex["dst_of"], dst_of) and np.array_equal(ex["size"], size)
+    assert np.array_equal(ex["kept_idx"], kept)
+    xm = ctx.merge(plan, x)
+    ctx.poll()
+    ref_m = O.merge(x64, dst_of, ctx.n_merged)
+    assert rel_err(to_f64(xm), ref_m) <= bf16_bound(ref_m)
+    plan.destroy()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ a6 / a10 merge, unmerge
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], ODD, MID], ids=lambda w: w.name)
 def test_merge_unmerge_with_oracle_plan(lib, wl):
