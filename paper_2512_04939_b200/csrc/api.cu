@@ -46,7 +46,7 @@ litevggt_status compute_sizes(const litevggt_config& c, Sizes* out) {
   z.frames = c.frames; z.grid_h = c.grid_h; z.grid_w = c.grid_w; z.n_special = c.n_special;
   z.dim = c.dim; z.heads = c.heads;
   const long long p = (long long)c.grid_h * c.grid_w;
-  if (p > 8192 || c.grid_w > 64) return LITEVGGT_ERR_BAD_CONFIG;  // the Var map kernel stages rows of <= 64 patches
+  if (p > 8192 || c.grid_w > 64) return LITEVGGT_ERR_BAD_CONFIG;  // the Var map kernel keeps per-row results of <= 64 columns in shared memory
   z.patches = (int)p;
   z.tokens_frame = (int)p + c.n_special;
   z.n_tokens = (long long)c.frames * z.tokens_frame;

@@ -137,10 +137,6 @@ bool resolve_encode_tiled(void** fn);
 bool make_tmap_bf16_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                        uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer);
 
-// same without swizzle: the box lands in shared memory as box_outer rows of box_inner elements
-bool make_tmap_bf16_2d_linear(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
-                              uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer);
-
 // scoring.cu
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches);
 cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var_parts, float* var,

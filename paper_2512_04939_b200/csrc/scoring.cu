@@ -98,145 +98,144 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 }
 
 // ----------------------------------------------------------------------------------------
-// Var map.  One CTA per (frame, grid row, quarter of the channels).  A single thread issues
-// two or three TMA loads - the 256-channel slices of the (clipped) 3 grid rows around the
-// CTA's row - so the whole 57 KB working set of the CTA is in flight at once; with several
-// CTAs per SM that is what keeps HBM busy.  Thread t then owns channels 2(t%128), 2(t%128)+1
-// and slides along its quarter of the row: per column it forms the sums of x - x0 and (x - x0)^2 over the window rows
-// (x0 = the row's first token, per channel, which removes a common offset before squaring),
-// a window is the sum of up to three columns, and the population variance follows as
-// E[d^2] - E[d]^2 in fp32.  The per-position sums over the CTA's 256 channels are reduced in
-// a fixed order and written to this quarter's plane; a second tiny kernel adds the four
-// planes in a fixed order, so the map is deterministic.
-constexpr int kVarThreads = 512;   // 128 channel pairs x 4 segments of the row
-constexpr int kVarSegments = kVarThreads / 128;
-constexpr int kVarChannels = 256;  // per CTA
+// Var map.  Summed over the channels, the population variance of a window W of n tokens is
+//     sum_c Var_c = (1/n) sum_{j in W} |d_j|^2  -  (1/n^2) sum_c (sum_{j in W} d_jc)^2,   d_j = x_j - x0,
+// for any fixed x0 (here the frame's first patch token, which takes a common offset out before
+// anything is squared).  So only the per-channel box sums of d are needed, plus a box sum of the
+// scalar |d_j|^2 - not a second per-channel box filter - and every token is read and unpacked once.
+//
+// A warp owns 16 channels of a block of 30 grid rows (+ one halo row on either side): lane = grid
+// row, and the warp walks along the row, one grid column per step.  Per step a lane loads its token's
+// 16 channels (32 bytes), forms d and |d|^2, gets the vertical 3-sums from its neighbour lanes by
+// shuffle, and keeps the last three columns of those in registers, from which the window sums of the
+// column before follow.  There is no barrier inside the walk.  A warp makes four such passes (64
+// channels), adding its results up in its own shared-memory rows; the four warps of a CTA cover a
+// quarter of the channels and are added in a fixed order into that quarter's plane, and
+// var_sum_kernel adds the four planes, so the map is deterministic.
+#ifndef LV_VAR_OCC
+#define LV_VAR_OCC 4
+#endif
+constexpr int kVarThreads = 128;
+constexpr int kVarWarps = kVarThreads / 32;
+constexpr int kVarChannels = 256;     // per CTA
+constexpr int kVarPassChannels = 16;  // per warp pass
+constexpr int kVarRowsPerBlock = 30;
 constexpr int kVarMaxW = 64;
 
-struct VarControl {
-  uint64_t bar;
-  uint32_t abort_flag;
-  uint32_t landed;
+struct VarColumn {
+  float s[kVarPassChannels];  // vertical 3-sum of d, per channel
+  float q;                    // vertical 3-sum of |d|^2
 };
-// dynamic shared memory: [control, 128 B][tile: nr x grid_w x 256 bf16][partial: grid_w x 32 fp32]
-__host__ __device__ inline size_t var_smem_bytes(int grid_w) {
-  return 128 + (size_t)3 * grid_w * kVarChannels * 2 + (size_t)grid_w * 32 * sizeof(float) + 128;
-}
 
-__global__ void __launch_bounds__(kVarThreads)
-var_map_kernel(const __grid_constant__ CUtensorMap tmap_x, float* __restrict__ var_parts, int frames, int grid_h,
-               int grid_w, int n_special, uint32_t* status) {
-  extern __shared__ uint8_t var_smem_raw[];
-  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(var_smem_raw) + 127) & ~uintptr_t(127));
-  VarControl* ctrl = reinterpret_cast<VarControl*>(base);
-  uint8_t* tile = base + 128;
-  const uint32_t row_bytes = (uint32_t)grid_w * kVarChannels * 2;  // one grid row of 256-channel slices
-  float* partial = reinterpret_cast<float*>(tile + 3 * (size_t)row_bytes);  // [grid_w][32]
-  const int quarter = blockIdx.x, py = blockIdx.y, f = blockIdx.z;
+__global__ void __launch_bounds__(kVarThreads, LV_VAR_OCC)
+var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var_parts, int frames, int grid_h, int grid_w,
+               int n_special) {
+  __shared__ float acc[kVarWarps][32][kVarMaxW + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quarter = blockIdx.x, f = blockIdx.z;
+  const int row = blockIdx.y * kVarRowsPerBlock - 1 + lane;  // lanes 0 and 31 are halo rows
+  const bool row_valid = row >= 0 && row < grid_h;
+  const bool emits = row_valid && lane >= 1 && lane <= kVarRowsPerBlock;
   const int tokens_frame = grid_h * grid_w + n_special;
-  const int r0 = py > 0 ? py - 1 : 0;
-  const int r1 = py < grid_h - 1 ? py + 1 : grid_h - 1;
-  const int nr = r1 - r0 + 1;
-  if (threadIdx.x == 0) {
-    mbar_init(&ctrl->bar, 1);
-    ctrl->abort_flag = 0;
-    mbar_fence_init();
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    mbar_expect_tx(&ctrl->bar, row_bytes * nr);
-    for (int r = 0; r < nr; ++r) {
-      const int token = f * tokens_frame + n_special + (r0 + r) * grid_w;
-      tma_load_2d(tile + (size_t)r * row_bytes, &tmap_x, &ctrl->bar, quarter * kVarChannels, token);
-    }
-  }
-  // Only the issuing thread polls the barrier; everyone else parks at the CTA barrier, which costs
-  // no issue slots (hundreds of polling threads would starve the CTAs that are computing).
-  if (threadIdx.x == 0) {
-    const WaitCtl ctl{&ctrl->abort_flag, status};
-    bool ok = mbar_wait(&ctrl->bar, 0, ctl);
-    if (!ok) {
-      // the copies are still in flight: they must finish before the shared memory is given up
-      const long long t0 = clock64();
-      while (!mbar_try_wait(&ctrl->bar, 0)) {
-        if (clock64() - t0 > kTimeoutCycles) break;
-      }
-    }
-    ctrl->landed = ok ? 1u : 0u;
-  }
-  __syncthreads();
-  const bool landed = ctrl->landed != 0u;
-  const int lane = threadIdx.x & 31;
-  if (landed) {
-    const int pair = threadIdx.x & 127, seg = threadIdx.x >> 7;
-    const int seg_len = (grid_w + kVarSegments - 1) / kVarSegments;
-    const int px_begin = seg * seg_len, px_end = min(grid_w, px_begin + seg_len);
-    const uint32_t* words = reinterpret_cast<const uint32_t*>(tile) + pair;  // this thread's channel pair
-    const int pitch = kVarChannels / 2;   // 32-bit words per token slice
-    const int row_words = grid_w * pitch; // per grid row
-    const uint32_t w0 = words[(py - r0) * row_words];
-    const float2 x0 = make_float2(bf16_lo(w0), bf16_hi(w0));
-    const bool three = nr == 3;  // CTA-uniform
-    // column sums of d and d^2 over the window rows, for the two channels of this thread (packed)
-    auto column = [&](int px, float2& s1, float2& s2) {
-      if (px < 0 || px >= grid_w) {
-        s1 = s2 = make_float2(0.0f, 0.0f);
-        return;
-      }
-      const uint32_t* p = words + px * pitch;
-      const uint32_t wa = p[0], wb = p[row_words];
-      const float2 da = make_float2(bf16_lo(wa) - x0.x, bf16_hi(wa) - x0.y);
-      const float2 db = make_float2(bf16_lo(wb) - x0.x, bf16_hi(wb) - x0.y);
-      s1 = __fadd2_rn(da, db);
-      s2 = __ffma2_rn(db, db, __fmul2_rn(da, da));
-      if (three) {
-        const uint32_t wc = p[2 * row_words];
-        const float2 dc = make_float2(bf16_lo(wc) - x0.x, bf16_hi(wc) - x0.y);
-        s1 = __fadd2_rn(s1, dc);
-        s2 = __ffma2_rn(dc, dc, s2);
-      }
-    };
-    const float inv_edge = 1.0f / (float)(nr * (grid_w > 1 ? 2 : 1)), inv_mid = 1.0f / (float)(nr * 3);
-    // one output position from the three column sums around it
-    auto emit = [&](int px, const float2& a1, const float2& a2, const float2& b1, const float2& b2, const float2& c1,
-                    const float2& c2) {
-      const float inv_n = (px == 0 || px == grid_w - 1) ? inv_edge : inv_mid;
-      const float2 inv2 = make_float2(inv_n, inv_n);
-      const float2 mean = __fmul2_rn(__fadd2_rn(__fadd2_rn(a1, b1), c1), inv2);
-      const float2 msq = __fmul2_rn(__fadd2_rn(__fadd2_rn(a2, b2), c2), inv2);
-      const float2 v = __ffma2_rn(make_float2(-mean.x, -mean.y), mean, msq);
-      float tot = fmaxf(v.x, 0.0f) + fmaxf(v.y, 0.0f);
-      // fixed-order partial reduction over groups of four lanes
-      tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-      tot += __shfl_xor_sync(0xffffffffu, tot, 2);
-      if ((lane & 3) == 0) partial[px * 32 + (pair >> 2)] = tot;
-    };
-    float2 a1, a2, b1, b2, c1, c2;
-    column(px_begin - 1, a1, a2);
-    column(px_begin, b1, b2);
-    // three positions per trip, so the column sums rotate through fixed registers
-    for (int px = px_begin; px < px_end; px += 3) {
-      column(px + 1, c1, c2);
-      emit(px, a1, a2, b1, b2, c1, c2);
-      if (px + 1 < px_end) {
-        column(px + 2, a1, a2);
-        emit(px + 1, b1, b2, c1, c2, a1, a2);
-      }
-      if (px + 2 < px_end) {
-        column(px + 3, b1, b2);
-        emit(px + 2, c1, c2, a1, a2, b1, b2);
-      }
-    }
-  }
-  __syncthreads();
-  if (!landed) return;
-  const int warp = threadIdx.x >> 5;
-  float* out = var_parts + ((size_t)quarter * frames + f) * grid_h * grid_w + (size_t)py * grid_w;
-  for (int px = warp; px < grid_w; px += kVarThreads / 32) {
-    float acc = partial[px * 32 + lane];
+  const __nv_bfloat16* frame = x + ((size_t)f * tokens_frame + n_special) * 1024;
+  const float inv_rows = 1.0f / (float)(1 + (row > 0 ? 1 : 0) + (row < grid_h - 1 ? 1 : 0));
+
+  for (int pass = 0; pass < kVarChannels / kVarWarps / kVarPassChannels; ++pass) {
+    // In one pass the four warps take the four 32-byte sectors of the same 128-byte lines, so a line
+    // comes from HBM once and the other three warps find it in cache.
+    const int ch = quarter * kVarChannels + (pass * kVarWarps + warp) * kVarPassChannels;
+    float x0[kVarPassChannels];
+    {
+      const uint4* p0 = reinterpret_cast<const uint4*>(frame + ch);
+      const uint4 a = __ldg(p0), b = __ldg(p0 + 1);
+      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) out[px] = acc;
+      for (int i = 0; i < 8; ++i) {
+        x0[2 * i] = bf16_lo(w[i]);
+        x0[2 * i + 1] = bf16_hi(w[i]);
+      }
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(frame + (size_t)(row_valid ? row : 0) * grid_w * 1024 + ch);
+    // one column: this lane's token -> d, |d|^2 -> vertical sums over the lanes above and below
+    auto column = [&](const uint4& a, const uint4& b, bool present, VarColumn& out) {
+      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      float d[kVarPassChannels];
+      float q = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        d[2 * i] = present ? bf16_lo(w[i]) - x0[2 * i] : 0.0f;
+        d[2 * i + 1] = present ? bf16_hi(w[i]) - x0[2 * i + 1] : 0.0f;
+        q = fmaf(d[2 * i], d[2 * i], q);
+        q = fmaf(d[2 * i + 1], d[2 * i + 1], q);
+      }
+      // lanes outside the grid hold zeros, so the clipped window needs no special case; lane 0 has
+      // no lane above it and lane 31 none below (their own results are never emitted)
+#pragma unroll
+      for (int i = 0; i < kVarPassChannels; ++i) {
+        const float up = __shfl_up_sync(0xffffffffu, d[i], 1), dn = __shfl_down_sync(0xffffffffu, d[i], 1);
+        out.s[i] = d[i] + (lane > 0 ? up : 0.0f) + (lane < 31 ? dn : 0.0f);
+      }
+      const float up = __shfl_up_sync(0xffffffffu, q, 1), dn = __shfl_down_sync(0xffffffffu, q, 1);
+      out.q = q + (lane > 0 ? up : 0.0f) + (lane < 31 ? dn : 0.0f);
+    };
+    // window of grid column px = columns l, m, r (absent ones are all-zero)
+    auto emit = [&](int px, const VarColumn& l, const VarColumn& m, const VarColumn& r) {
+      float m2 = 0.0f;
+#pragma unroll
+      for (int i = 0; i < kVarPassChannels; ++i) {
+        const float t = l.s[i] + m.s[i] + r.s[i];
+        m2 = fmaf(t, t, m2);
+      }
+      const float inv_n = inv_rows * ((px > 0 && px < grid_w - 1) ? (1.0f / 3.0f) : (grid_w > 1 ? 0.5f : 1.0f));
+      const float v = (l.q + m.q + r.q) * inv_n - m2 * inv_n * inv_n;
+      if (emits) {
+        float* slot = &acc[warp][lane][px];
+        *slot = pass == 0 ? v : *slot + v;
+      }
+    };
+    VarColumn ca, cb, cc;
+#pragma unroll
+    for (int i = 0; i < kVarPassChannels; ++i) ca.s[i] = 0.0f;
+    ca.q = 0.0f;
+    // the raw tokens of the next three columns are in flight ahead of the one being worked on; with
+    // three buffers and three columns per trip every buffer keeps its role
+    uint4 r0a = make_uint4(0, 0, 0, 0), r0b = r0a, r1a = r0a, r1b = r0a, r2a = r0a, r2b = r0a;
+    auto fetch = [&](int px, uint4& a, uint4& b) {  // token (row, px); a column is 128 x 16 bytes further on
+      if (row_valid && px < grid_w) {
+        a = __ldg(src + (size_t)px * 128);
+        b = __ldg(src + (size_t)px * 128 + 1);
+      }
+    };
+    {
+      uint4 a = r0a, b = r0b;
+      fetch(0, a, b);
+      fetch(1, r0a, r0b);
+      fetch(2, r1a, r1b);
+      fetch(3, r2a, r2b);
+      column(a, b, row_valid, cb);
+    }
+    // one grid column: finish the sums of column px + 1 (raw in ra, rb, refilled with column px + 4),
+    // emit the window around column px
+    auto step = [&](int px, uint4& ra, uint4& rb, const VarColumn& l, const VarColumn& m, VarColumn& r) {
+      const uint4 a = ra, b = rb;
+      fetch(px + 4, ra, rb);
+      column(a, b, row_valid && px + 1 < grid_w, r);
+      emit(px, l, m, r);
+    };
+    for (int px = 0; px < grid_w; px += 3) {
+      step(px, r0a, r0b, ca, cb, cc);
+      if (px + 1 < grid_w) step(px + 1, r1a, r1b, cb, cc, ca);
+      if (px + 2 < grid_w) step(px + 2, r2a, r2b, cc, ca, cb);
+    }
+  }
+  __syncthreads();
+  // rows of this block, all columns: the four warps' partial sums in a fixed order
+  const int r0 = blockIdx.y * kVarRowsPerBlock;
+  const int n_rows = min(kVarRowsPerBlock, grid_h - r0);
+  float* out = var_parts + ((size_t)quarter * frames + f) * grid_h * grid_w + (size_t)r0 * grid_w;
+  for (int i = threadIdx.x; i < n_rows * grid_w; i += kVarThreads) {
+    const int r = i / grid_w, px = i - r * grid_w;
+    out[i] = ((acc[0][r + 1][px] + acc[1][r + 1][px]) + acc[2][r + 1][px]) + acc[3][r + 1][px];
   }
 }
 
@@ -248,15 +247,9 @@ __global__ void var_sum_kernel(const float* __restrict__ parts, float* __restric
 cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var_parts, float* var,
                            cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
-  CUtensorMap tmap;
-  if (!make_tmap_bf16_2d_linear(ctx->encode_tiled, &tmap, x, 1024, (uint64_t)z.n_tokens, 1024, kVarChannels,
-                                (uint32_t)z.grid_w))
-    return cudaErrorInvalidValue;
-  const int smem = (int)var_smem_bytes(z.grid_w);
-  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  var_map_kernel<<<dim3(4, z.grid_h, z.frames), kVarThreads, smem, s>>>(tmap, var_parts, z.frames, z.grid_h, z.grid_w,
-                                                                        z.n_special, ctx->ws.status);
+  const unsigned row_blocks = (unsigned)((z.grid_h + kVarRowsPerBlock - 1) / kVarRowsPerBlock);
+  var_map_kernel<<<dim3(4, row_blocks, z.frames), kVarThreads, 0, s>>>(x, var_parts, z.frames, z.grid_h, z.grid_w,
+                                                                      z.n_special);
   ++*launches;
   const long long count = (long long)z.frames * z.patches;
   var_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(var_parts, var, count);

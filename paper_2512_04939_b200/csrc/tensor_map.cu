@@ -37,10 +37,4 @@ bool make_tmap_bf16_2d(void* encode_fn, CUtensorMap* out, const void* base, uint
                         CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-bool make_tmap_bf16_2d_linear(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
-                              uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer) {
-  return encode_bf16_2d(encode_fn, out, base, inner, outer, pitch_elems, box_inner, box_outer,
-                        CU_TENSOR_MAP_SWIZZLE_NONE);
-}
-
 }  // namespace lv
