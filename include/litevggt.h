@@ -59,7 +59,7 @@ enum {
 typedef struct {
   int32_t frames;             /* F >= 1 */
   int32_t grid_h, grid_w;     /* patch grid; image is (14*grid_h) x (14*grid_w) pixels; grid_w <= 64 */
-  int32_t patch_px;           /* 14 */
+  int32_t patch_px;           /* 14; at most 30 */
   int32_t n_special;          /* 5 (1 camera + 4 register tokens, ahead of the patches) */
   int32_t dim;                /* 1024 */
   int32_t heads;              /* 16 (head dim must be 64) */

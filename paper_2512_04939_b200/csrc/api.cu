@@ -41,7 +41,7 @@ litevggt_status compute_sizes(const litevggt_config& c, Sizes* out) {
   if (!(c.merge_ratio >= 0.0f && c.merge_ratio <= 1.0f)) return LITEVGGT_ERR_BAD_CONFIG;
   if (!(c.ga_keep_frac >= 0.0f && c.ga_keep_frac <= 1.0f)) return LITEVGGT_ERR_BAD_CONFIG;
   if (c.qkv_dtype != 0) return LITEVGGT_ERR_BAD_CONFIG;
-  if (c.patch_px > 32) return LITEVGGT_ERR_BAD_CONFIG;
+  if (c.patch_px > 30) return LITEVGGT_ERR_BAD_CONFIG;  // a patch and its two halo columns share a warp in the Grad map
   Sizes z;
   z.frames = c.frames; z.grid_h = c.grid_h; z.grid_w = c.grid_w; z.n_special = c.n_special;
   z.dim = c.dim; z.heads = c.heads;

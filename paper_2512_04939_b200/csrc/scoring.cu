@@ -8,14 +8,24 @@
 namespace lv {
 
 // ----------------------------------------------------------------------------------------
-// Grad map.  One CTA per (frame, patch row).  Phase 1: the 16 grey rows it needs (14 + one halo
-// row above and below, replicate padding) are staged in shared memory, one warp per image row,
-// two pixels per load when the width is even.  Phase 2: one thread per pixel column walks down
-// the 16 rows with the separable form of the Sobel pair - per row the horizontal difference
-// r - l and the horizontal smoothing l + 2c + r, kept for the last three rows - and adds up the
-// 14 magnitudes of its column.  Phase 3: one thread per patch adds its 14 column sums.  All sums
-// run in a fixed order.
-constexpr int kGradThreads = 256;
+// Grad map.  A warp owns a vertical strip of the image - as many whole patches as fit into 30 pixel
+// columns, plus one halo column on either side (lane = pixel column, replicate padding by clamping
+// the coordinate) - over a block of 7 patch rows, and walks down it one image row per step: three
+// coalesced 4-byte loads per lane (R, G, B), the grey value, its left and right neighbours by
+// shuffle, the separable Sobel pair (per row the horizontal difference r - l and the horizontal
+// smoothing l + 2c + r, kept for the last three rows), the magnitude, a running sum per column.  At
+// the bottom of a patch row the columns of a patch are added by a shuffle tree and one lane writes
+// the patch mean.  Rows are loaded three steps ahead (deeper measured slower); there is no shared
+// memory and no barrier.
+constexpr int kGradThreads = 128;
+#ifndef LV_GRAD_PATCH_ROWS
+#define LV_GRAD_PATCH_ROWS 7
+#endif
+#ifndef LV_GRAD_AHEAD
+#define LV_GRAD_AHEAD 3
+#endif
+constexpr int kGradPatchRows = LV_GRAD_PATCH_ROWS;  // patch rows per warp
+constexpr int kGradAhead = LV_GRAD_AHEAD;           // image rows in flight
 
 __device__ __forceinline__ float sqrt_approx(float x) {
   float y;
@@ -25,74 +35,83 @@ __device__ __forceinline__ float sqrt_approx(float x) {
 
 __global__ void __launch_bounds__(kGradThreads)
 grad_map_kernel(const float* __restrict__ images, float* __restrict__ grad, int grid_h, int grid_w, int patch) {
-  extern __shared__ float grey[];  // [(patch+2)][w+2], then [w] column sums
-  const int f = blockIdx.y;
-  const int py = blockIdx.x;
-  const int h = grid_h * patch, w = grid_w * patch;
-  const int pitch = w + 2;
-  const int rows = patch + 2;
-  float* colsum = grey + rows * pitch;
-  const size_t plane = (size_t)h * w;
-  const float* img = images + (size_t)f * 3 * plane;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int r = warp; r < rows; r += kGradThreads / 32) {
-    int y = py * patch - 1 + r;
+  const int pps = 30 / patch;  // patches per strip (patch <= 30)
+  const int strips = (grid_w + pps - 1) / pps;
+  const int strip = blockIdx.x * (kGradThreads / 32) + warp;
+  if (strip >= strips) return;  // whole warp; nothing below synchronises across warps
+  const int f = blockIdx.z;
+  const int pr0 = blockIdx.y * kGradPatchRows;
+  const int pr1 = min(grid_h, pr0 + kGradPatchRows);
+  const int h = grid_h * patch, w = grid_w * patch;
+  const size_t plane = (size_t)h * w;
+  int x = strip * pps * patch - 1 + lane;
+  x = x < 0 ? 0 : (x >= w ? w - 1 : x);
+  const float* col = images + (size_t)f * 3 * plane + x;
+  // lanes 1 .. pps * patch carry the strip's own pixel columns
+  const bool own = lane >= 1 && lane <= pps * patch;
+  const int seg = own ? (lane - 1) / patch : 0;
+  const int in_seg = own ? (lane - 1) - seg * patch : patch;
+  const int patch_x = strip * pps + seg;
+  const bool writer = own && in_seg == 0 && patch_x < grid_w;
+
+  const float inv_area = 1.0f / (float)(patch * patch);
+  const int y_first = pr0 * patch - 1;             // halo row above (clamped when it is outside)
+  const int count = (pr1 - pr0) * patch + 2;       // rows visited, halo rows included
+  float q[kGradAhead][3];
+  auto load_row = [&](int i, float (&dst)[3]) {
+    int y = y_first + i;
     y = y < 0 ? 0 : (y >= h ? h - 1 : y);
-    const float* p0 = img + (size_t)y * w;
-    float* g = grey + r * pitch + 1;
-    if ((w & 1) == 0) {  // rows are 8-byte aligned
-      const float2* q0 = reinterpret_cast<const float2*>(p0);
-      const float2* q1 = reinterpret_cast<const float2*>(p0 + plane);
-      const float2* q2 = reinterpret_cast<const float2*>(p0 + 2 * plane);
-      const int half_w = w >> 1;
-#pragma unroll 4
-      for (int xh = lane; xh < half_w; xh += 32) {
-        const float2 a = __ldg(q0 + xh), b = __ldg(q1 + xh), c = __ldg(q2 + xh);
-        g[2 * xh] = (a.x + b.x + c.x) / 3.0f;
-        g[2 * xh + 1] = (a.y + b.y + c.y) / 3.0f;
+    const float* p = col + (size_t)y * w;
+    dst[0] = __ldg(p);
+    dst[1] = __ldg(p + plane);
+    dst[2] = __ldg(p + 2 * plane);
+  };
+#pragma unroll
+  for (int k = 0; k < kGradAhead; ++k)
+    if (k < count) load_row(k, q[k]);
+  float d0 = 0.0f, s0 = 0.0f, d1 = 0.0f, s1 = 0.0f, acc = 0.0f;
+  int rows_done = 0, pr = pr0;
+  for (int i0 = 0; i0 < count; i0 += kGradAhead) {
+#pragma unroll
+    for (int k = 0; k < kGradAhead; ++k) {
+      const int i = i0 + k;
+      if (i >= count) break;  // warp-uniform
+      const float g = (q[k][0] + q[k][1] + q[k][2]) * (1.0f / 3.0f);
+      if (i + kGradAhead < count) load_row(i + kGradAhead, q[k]);
+      const float l = __shfl_up_sync(0xffffffffu, g, 1), r = __shfl_down_sync(0xffffffffu, g, 1);
+      const float d = r - l, s = fmaf(2.0f, g, l + r);
+      if (i >= 2) {  // rows i-2, i-1, i are in hand: the pixel of row i-1
+        const float gx = fmaf(2.0f, d1, d0 + d);
+        const float gy = s - s0;
+        acc += sqrt_approx(fmaf(gx, gx, gy * gy));
+        if (++rows_done == patch) {
+          // bottom of a patch row: add the columns of each patch, lowest lane of the patch writes
+          float v = own ? acc : 0.0f;
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            const float t = __shfl_down_sync(0xffffffffu, v, off);
+            if (in_seg + off < patch) v += t;
+          }
+          if (writer) grad[((size_t)f * grid_h + pr) * grid_w + patch_x] = v * inv_area;
+          acc = 0.0f;
+          rows_done = 0;
+          ++pr;
+        }
       }
-    } else {
-#pragma unroll 4
-      for (int x = lane; x < w; x += 32) g[x] = (__ldg(p0 + x) + __ldg(p0 + plane + x) + __ldg(p0 + 2 * plane + x)) / 3.0f;
+      d0 = d1; s0 = s1; d1 = d; s1 = s;
     }
-    __syncwarp();
-    if (lane == 0) {
-      g[-1] = g[0];
-      g[w] = g[w - 1];
-    }
-  }
-  __syncthreads();
-  for (int col = threadIdx.x; col < w; col += kGradThreads) {
-    const float* p = grey + col;  // p[0], p[1], p[2] = left, centre, right of this column in row 0
-    float d0 = p[2] - p[0], s0 = fmaf(2.0f, p[1], p[0] + p[2]);
-    p += pitch;
-    float d1 = p[2] - p[0], s1 = fmaf(2.0f, p[1], p[0] + p[2]);
-    float acc = 0.0f;
-    for (int r = 0; r < patch; ++r) {
-      p += pitch;
-      const float d2 = p[2] - p[0], s2 = fmaf(2.0f, p[1], p[0] + p[2]);
-      const float gx = fmaf(2.0f, d1, d0 + d2);
-      const float gy = s2 - s0;
-      acc += sqrt_approx(fmaf(gx, gx, gy * gy));
-      d0 = d1; s0 = s1; d1 = d2; s1 = s2;
-    }
-    colsum[col] = acc;
-  }
-  __syncthreads();
-  for (int px = threadIdx.x; px < grid_w; px += kGradThreads) {
-    float acc = 0.0f;
-    for (int c = 0; c < patch; ++c) acc += colsum[px * patch + c];
-    grad[((size_t)f * grid_h + py) * grid_w + px] = acc / (float)(patch * patch);
   }
 }
 
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
   const int patch = ctx->cfg.patch_px;
-  const size_t smem = ((size_t)(patch + 2) * (z.grid_w * patch + 2) + (size_t)z.grid_w * patch) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(grad_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  grad_map_kernel<<<dim3(z.grid_h, z.frames), kGradThreads, smem, s>>>(images, grad, z.grid_h, z.grid_w, patch);
+  const int pps = 30 / patch;
+  const int strips = (z.grid_w + pps - 1) / pps;
+  const dim3 grid((unsigned)((strips + kGradThreads / 32 - 1) / (kGradThreads / 32)),
+                  (unsigned)((z.grid_h + kGradPatchRows - 1) / kGradPatchRows), (unsigned)z.frames);
+  grad_map_kernel<<<grid, kGradThreads, 0, s>>>(images, grad, z.grid_h, z.grid_w, patch);
   ++*launches;
   return cudaGetLastError();
 }
