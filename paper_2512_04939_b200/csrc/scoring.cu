@@ -121,18 +121,26 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 //     sum_c Var_c = (1/n) sum_{j in W} |d_j|^2  -  (1/n^2) sum_c (sum_{j in W} d_jc)^2,   d_j = x_j - x0,
 // for any fixed x0 (here the frame's first patch token, which takes a common offset out before
 // anything is squared).  So only the per-channel box sums of d are needed, plus a box sum of the
-// scalar |d_j|^2 - not a second per-channel box filter - and every token is read and unpacked once.
+// scalar |d_j|^2 - not a second per-channel box filter.
 //
-// A warp owns 16 channels of a block of 30 grid rows (+ one halo row on either side): lane = grid
-// row, and the warp walks along the row, one grid column per step.  Per step a lane loads its token's
-// 16 channels (32 bytes), forms d and |d|^2, gets the vertical 3-sums from its neighbour lanes by
-// shuffle, and keeps the last three columns of those in registers, from which the window sums of the
-// column before follow.  There is no barrier inside the walk.  A warp makes four such passes (64
-// channels), adding its results up in its own shared-memory rows; the four warps of a CTA cover a
-// quarter of the channels and are added in a fixed order into that quarter's plane, and
-// var_sum_kernel adds the four planes, so the map is deterministic.
+// A warp owns 16 channels of a block of 30 grid rows (+ one halo row on either side) and walks along
+// the rows, one grid column per step.  The column's 32 tokens (32 bytes each) arrive in the warp's own
+// ring in shared memory by asynchronous copies, two lanes per token, kVarDepth columns ahead; rows
+// outside the grid are filled with x0, so they contribute d = 0 and the clipped window needs no
+// special case.  Lane = grid row: it reads its own token and the ones above and below from the ring
+// (48-byte row pitch: conflict-free 16-byte reads), forms the vertical sums of d and of |d|^2, and
+// keeps the last three columns in registers, from which the window sums of the column before follow.
+// Scattered 16-byte global loads and two shuffles per channel cost this kernel's first version
+// (lane loads its own token, neighbours by shuffle) three times the L1 wavefronts.  No barrier
+// inside the walk; only __syncwarp around the ring.  A warp makes four such passes (64 channels),
+// adding its results up in its own shared-memory rows; the four warps of a CTA cover a quarter of
+// the channels and are added in a fixed order into that quarter's plane, and var_sum_kernel adds the
+// four planes, so the map is deterministic.
 #ifndef LV_VAR_OCC
 #define LV_VAR_OCC 4
+#endif
+#ifndef LV_VAR_DEPTH
+#define LV_VAR_DEPTH 4
 #endif
 constexpr int kVarThreads = 128;
 constexpr int kVarWarps = kVarThreads / 32;
@@ -140,121 +148,171 @@ constexpr int kVarChannels = 256;     // per CTA
 constexpr int kVarPassChannels = 16;  // per warp pass
 constexpr int kVarRowsPerBlock = 30;
 constexpr int kVarMaxW = 64;
+constexpr int kVarDepth = LV_VAR_DEPTH;  // grid columns in flight
+constexpr int kVarRowPitch = 48;         // bytes per token in the ring: 32 of data + 16 against bank conflicts
+constexpr int kVarSlotBytes = 32 * kVarRowPitch;
+// dynamic shared memory per warp: the ring [depth][32 rows][48 B], then this warp's results
+// [32 lanes][grid_w + 1]
+__host__ __device__ inline size_t var_warp_smem_bytes(int grid_w) {
+  return (size_t)kVarDepth * kVarSlotBytes + (size_t)32 * (grid_w + 1) * sizeof(float);
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+}
 
 struct VarColumn {
-  float s[kVarPassChannels];  // vertical 3-sum of d, per channel
-  float q;                    // vertical 3-sum of |d|^2
+  float2 s[kVarPassChannels / 2];  // vertical 3-sum of d, per channel (pairs: packed fp32 arithmetic)
+  float q;                         // vertical 3-sum of |d|^2
 };
 
 __global__ void __launch_bounds__(kVarThreads, LV_VAR_OCC)
 var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var_parts, int frames, int grid_h, int grid_w,
                int n_special) {
-  __shared__ float acc[kVarWarps][32][kVarMaxW + 1];
+  extern __shared__ __align__(16) uint8_t var_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t warp_bytes = var_warp_smem_bytes(grid_w);
+  uint8_t* ring = var_smem + warp * warp_bytes;
+  const int acc_pitch = grid_w + 1;
+  float* acc = reinterpret_cast<float*>(ring + kVarDepth * kVarSlotBytes) + lane * acc_pitch;  // this lane's results
   const int quarter = blockIdx.x, f = blockIdx.z;
-  const int row = blockIdx.y * kVarRowsPerBlock - 1 + lane;  // lanes 0 and 31 are halo rows
+  const int row0 = blockIdx.y * kVarRowsPerBlock - 1;  // grid row of lane 0 (a halo row)
+  const int row = row0 + lane;
   const bool row_valid = row >= 0 && row < grid_h;
   const bool emits = row_valid && lane >= 1 && lane <= kVarRowsPerBlock;
   const int tokens_frame = grid_h * grid_w + n_special;
   const __nv_bfloat16* frame = x + ((size_t)f * tokens_frame + n_special) * 1024;
   const float inv_rows = 1.0f / (float)(1 + (row > 0 ? 1 : 0) + (row < grid_h - 1 ? 1 : 0));
+  // as a copier, this lane moves 16 bytes of two tokens per column: rows row0 + lane/2 and + 16
+  const int half = lane & 1;
+  const int crow_a = row0 + (lane >> 1), crow_b = crow_a + 16;
+  const bool cvalid_a = crow_a >= 0 && crow_a < grid_h, cvalid_b = crow_b >= 0 && crow_b < grid_h;
+  // lanes 0 and 31 have no row above / below in the ring: they read their own row instead; what they
+  // compute is never emitted
+  const int up = lane > 0 ? lane - 1 : lane, dn = lane < 31 ? lane + 1 : lane;
 
   for (int pass = 0; pass < kVarChannels / kVarWarps / kVarPassChannels; ++pass) {
     // In one pass the four warps take the four 32-byte sectors of the same 128-byte lines, so a line
     // comes from HBM once and the other three warps find it in cache.
     const int ch = quarter * kVarChannels + (pass * kVarWarps + warp) * kVarPassChannels;
-    float x0[kVarPassChannels];
+    const __nv_bfloat16* x0_ptr = frame + ch;  // first patch token of the frame, this pass's channels
+    float2 x0[kVarPassChannels / 2], x0_3[kVarPassChannels / 2];
     {
-      const uint4* p0 = reinterpret_cast<const uint4*>(frame + ch);
+      const uint4* p0 = reinterpret_cast<const uint4*>(x0_ptr);
       const uint4 a = __ldg(p0), b = __ldg(p0 + 1);
       const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        x0[2 * i] = bf16_lo(w[i]);
-        x0[2 * i + 1] = bf16_hi(w[i]);
+        x0[i] = make_float2(bf16_lo(w[i]), bf16_hi(w[i]));
+        x0_3[i] = make_float2(-3.0f * x0[i].x, -3.0f * x0[i].y);
       }
     }
-    const uint4* src = reinterpret_cast<const uint4*>(frame + (size_t)(row_valid ? row : 0) * grid_w * 1024 + ch);
-    // one column: this lane's token -> d, |d|^2 -> vertical sums over the lanes above and below
-    auto column = [&](const uint4& a, const uint4& b, bool present, VarColumn& out) {
+    const __nv_bfloat16* src_a = cvalid_a ? frame + (size_t)crow_a * grid_w * 1024 + ch + half * 8 : nullptr;
+    const __nv_bfloat16* src_b = cvalid_b ? frame + (size_t)crow_b * grid_w * 1024 + ch + half * 8 : nullptr;
+    // column px into its slot of the ring; one copy group per column (empty past the last column), so
+    // the number of groups still pending tells which columns have landed
+    auto fetch = [&](int px) {
+      if (px < grid_w) {
+        uint8_t* slot = ring + (px % kVarDepth) * kVarSlotBytes + half * 16;
+        cp_async16(slot + (lane >> 1) * kVarRowPitch, src_a != nullptr ? src_a + (size_t)px * 1024 : x0_ptr + half * 8);
+        cp_async16(slot + ((lane >> 1) + 16) * kVarRowPitch,
+                   src_b != nullptr ? src_b + (size_t)px * 1024 : x0_ptr + half * 8);
+      }
+      cp_async_commit();
+    };
+#pragma unroll
+    for (int k = 0; k < kVarDepth; ++k) fetch(k);
+    // the 16 channels of one token of the slot, as 8 pairs
+    auto load_x = [&](const uint8_t* slot, int r, float2 (&v)[kVarPassChannels / 2]) {
+      const uint4* p = reinterpret_cast<const uint4*>(slot + r * kVarRowPitch);
+      const uint4 a = p[0], b = p[1];
       const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-      float d[kVarPassChannels];
-      float q = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        d[2 * i] = present ? bf16_lo(w[i]) - x0[2 * i] : 0.0f;
-        d[2 * i + 1] = present ? bf16_hi(w[i]) - x0[2 * i + 1] : 0.0f;
-        q = fmaf(d[2 * i], d[2 * i], q);
-        q = fmaf(d[2 * i + 1], d[2 * i + 1], q);
-      }
-      // lanes outside the grid hold zeros, so the clipped window needs no special case; lane 0 has
-      // no lane above it and lane 31 none below (their own results are never emitted)
+      for (int i = 0; i < 8; ++i) v[i] = make_float2(bf16_lo(w[i]), bf16_hi(w[i]));
+    };
+    // one grid column: vertical sums over this lane's row and the rows above and below, then the
+    // slot goes back to the copiers.  Rows outside the grid hold x0, so the sum of d over the three
+    // rows is always (sum of x) - 3 x0.
+    auto take = [&](int c, VarColumn& out) {
+      if (c < grid_w) {
+        cp_async_wait<kVarDepth - 1>();  // all but the newest kVarDepth - 1 groups: column c has landed
+        __syncwarp();                     // ... for every lane's copies
+        const uint8_t* slot = ring + (c % kVarDepth) * kVarSlotBytes;
+        float2 v[kVarPassChannels / 2];
+        load_x(slot, lane, v);
+        float2 q2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int i = 0; i < kVarPassChannels; ++i) {
-        const float up = __shfl_up_sync(0xffffffffu, d[i], 1), dn = __shfl_down_sync(0xffffffffu, d[i], 1);
-        out.s[i] = d[i] + (lane > 0 ? up : 0.0f) + (lane < 31 ? dn : 0.0f);
+        for (int i = 0; i < kVarPassChannels / 2; ++i) {
+          const float2 d = __fadd2_rn(v[i], make_float2(-x0[i].x, -x0[i].y));
+          q2 = __ffma2_rn(d, d, q2);
+          out.s[i] = __fadd2_rn(v[i], x0_3[i]);
+        }
+        load_x(slot, up, v);
+#pragma unroll
+        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = __fadd2_rn(out.s[i], v[i]);
+        load_x(slot, dn, v);
+#pragma unroll
+        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = __fadd2_rn(out.s[i], v[i]);
+        const float q = q2.x + q2.y;
+        const float q_up = __shfl_up_sync(0xffffffffu, q, 1), q_dn = __shfl_down_sync(0xffffffffu, q, 1);
+        out.q = q + (lane > 0 ? q_up : 0.0f) + (lane < 31 ? q_dn : 0.0f);
+        __syncwarp();  // every lane has read the slot
+      } else {
+#pragma unroll
+        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = make_float2(0.0f, 0.0f);
+        out.q = 0.0f;
       }
-      const float up = __shfl_up_sync(0xffffffffu, q, 1), dn = __shfl_down_sync(0xffffffffu, q, 1);
-      out.q = q + (lane > 0 ? up : 0.0f) + (lane < 31 ? dn : 0.0f);
+      fetch(c + kVarDepth);
     };
     // window of grid column px = columns l, m, r (absent ones are all-zero)
     auto emit = [&](int px, const VarColumn& l, const VarColumn& m, const VarColumn& r) {
-      float m2 = 0.0f;
+      float2 m2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int i = 0; i < kVarPassChannels; ++i) {
-        const float t = l.s[i] + m.s[i] + r.s[i];
-        m2 = fmaf(t, t, m2);
+      for (int i = 0; i < kVarPassChannels / 2; ++i) {
+        const float2 t = __fadd2_rn(__fadd2_rn(l.s[i], m.s[i]), r.s[i]);
+        m2 = __ffma2_rn(t, t, m2);
       }
       const float inv_n = inv_rows * ((px > 0 && px < grid_w - 1) ? (1.0f / 3.0f) : (grid_w > 1 ? 0.5f : 1.0f));
-      const float v = (l.q + m.q + r.q) * inv_n - m2 * inv_n * inv_n;
-      if (emits) {
-        float* slot = &acc[warp][lane][px];
-        *slot = pass == 0 ? v : *slot + v;
-      }
+      const float v = (l.q + m.q + r.q) * inv_n - (m2.x + m2.y) * inv_n * inv_n;
+      if (emits) acc[px] = pass == 0 ? v : acc[px] + v;
     };
     VarColumn ca, cb, cc;
 #pragma unroll
-    for (int i = 0; i < kVarPassChannels; ++i) ca.s[i] = 0.0f;
+    for (int i = 0; i < kVarPassChannels / 2; ++i) ca.s[i] = make_float2(0.0f, 0.0f);
     ca.q = 0.0f;
-    // the raw tokens of the next three columns are in flight ahead of the one being worked on; with
-    // three buffers and three columns per trip every buffer keeps its role
-    uint4 r0a = make_uint4(0, 0, 0, 0), r0b = r0a, r1a = r0a, r1b = r0a, r2a = r0a, r2b = r0a;
-    auto fetch = [&](int px, uint4& a, uint4& b) {  // token (row, px); a column is 128 x 16 bytes further on
-      if (row_valid && px < grid_w) {
-        a = __ldg(src + (size_t)px * 128);
-        b = __ldg(src + (size_t)px * 128 + 1);
-      }
-    };
-    {
-      uint4 a = r0a, b = r0b;
-      fetch(0, a, b);
-      fetch(1, r0a, r0b);
-      fetch(2, r1a, r1b);
-      fetch(3, r2a, r2b);
-      column(a, b, row_valid, cb);
-    }
-    // one grid column: finish the sums of column px + 1 (raw in ra, rb, refilled with column px + 4),
-    // emit the window around column px
-    auto step = [&](int px, uint4& ra, uint4& rb, const VarColumn& l, const VarColumn& m, VarColumn& r) {
-      const uint4 a = ra, b = rb;
-      fetch(px + 4, ra, rb);
-      column(a, b, row_valid && px + 1 < grid_w, r);
-      emit(px, l, m, r);
-    };
+    take(0, cb);
+    // three columns per trip, so the column sums rotate through fixed registers
     for (int px = 0; px < grid_w; px += 3) {
-      step(px, r0a, r0b, ca, cb, cc);
-      if (px + 1 < grid_w) step(px + 1, r1a, r1b, cb, cc, ca);
-      if (px + 2 < grid_w) step(px + 2, r2a, r2b, cc, ca, cb);
+      take(px + 1, cc);
+      emit(px, ca, cb, cc);
+      if (px + 1 < grid_w) {
+        take(px + 2, ca);
+        emit(px + 1, cb, cc, ca);
+      }
+      if (px + 2 < grid_w) {
+        take(px + 3, cb);
+        emit(px + 2, cc, ca, cb);
+      }
     }
+    cp_async_wait<0>();
+    __syncwarp();
   }
   __syncthreads();
   // rows of this block, all columns: the four warps' partial sums in a fixed order
   const int r0 = blockIdx.y * kVarRowsPerBlock;
   const int n_rows = min(kVarRowsPerBlock, grid_h - r0);
   float* out = var_parts + ((size_t)quarter * frames + f) * grid_h * grid_w + (size_t)r0 * grid_w;
+  auto warp_acc = [&](int w, int lane_row, int px) {
+    return reinterpret_cast<const float*>(var_smem + w * warp_bytes + kVarDepth * kVarSlotBytes)[lane_row * acc_pitch + px];
+  };
   for (int i = threadIdx.x; i < n_rows * grid_w; i += kVarThreads) {
     const int r = i / grid_w, px = i - r * grid_w;
-    out[i] = ((acc[0][r + 1][px] + acc[1][r + 1][px]) + acc[2][r + 1][px]) + acc[3][r + 1][px];
+    out[i] = ((warp_acc(0, r + 1, px) + warp_acc(1, r + 1, px)) + warp_acc(2, r + 1, px)) + warp_acc(3, r + 1, px);
   }
 }
 
@@ -267,8 +325,11 @@ cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, floa
                            cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
   const unsigned row_blocks = (unsigned)((z.grid_h + kVarRowsPerBlock - 1) / kVarRowsPerBlock);
-  var_map_kernel<<<dim3(4, row_blocks, z.frames), kVarThreads, 0, s>>>(x, var_parts, z.frames, z.grid_h, z.grid_w,
-                                                                      z.n_special);
+  const int smem = (int)(kVarWarps * var_warp_smem_bytes(z.grid_w));
+  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  var_map_kernel<<<dim3(4, row_blocks, z.frames), kVarThreads, smem, s>>>(x, var_parts, z.frames, z.grid_h, z.grid_w,
+                                                                         z.n_special);
   ++*launches;
   const long long count = (long long)z.frames * z.patches;
   var_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(var_parts, var, count);
