@@ -200,7 +200,8 @@ litevggt_status litevggt_layernorm(litevggt_ctx* ctx, const void* x, int64_t row
 litevggt_status litevggt_frame_attn(litevggt_ctx* ctx, const void* x, const void* w_qkv, const void* b_qkv,
                                     const void* w_o, const void* b_o, const void* residual, void* y, void* stream);
 
-/* Transformer MLP: y = residual + gelu(x w1^T + b1) w2^T + b2 with the exact (erf) GELU.
+/* Transformer MLP: y = residual + gelu(x w1^T + b1) w2^T + b2 with the erf form of GELU, 0.5 x (1 + erf(x / sqrt 2))
+ * (erf by a rational approximation with absolute error below 1.5e-7, far under the bf16 rounding of the result).
  * x, residual (nullable), y: dev bf16 [rows, D], rows <= N; w1: dev bf16 [4D, D]; b1: dev bf16 [4D] or
  * NULL; w2: dev bf16 [D, 4D]; b2: dev bf16 [D] or NULL. */
 litevggt_status litevggt_mlp(litevggt_ctx* ctx, const void* x, int64_t rows, const void* w1, const void* b1,
