@@ -96,6 +96,26 @@ def test_var_map_and_partition(lib, wl):
     ctx.close()
 
 
+def test_scoring_maps_on_the_widest_grid(lib):
+    """Grid of 33 x 64 patches: the widest row the library accepts (the Var map's per-row results and
+    the Grad map's strips reach their limits), more than one block of 30 grid rows, and a frame whose
+    last strip holds two patches exactly."""
+    wl = Workload("WIDE", 2, 33, 64, 0.5, "polygons", 1, 6, 9000)
+    img = make_images(wl)
+    tok = make_tokens(wl, img)
+    ctx = _ctx(lib, wl)
+    grad = ctx.grad_map(img.cuda())
+    ref_grad = O.grad_map(img.numpy())
+    assert np.abs(to_f64(grad) - ref_grad).max() <= 1e-5 * max(ref_grad.max(), 1e-3)
+    plan = ctx.merge_plan(tok.cuda(), grad)
+    ctx.poll()
+    ex = ctx.plan_export(plan)
+    ref_var = O.var_map(to_f64(tok), wl.frames, wl.grid_h, wl.grid_w)
+    assert np.abs(ex["var"] - ref_var).max() <= 2e-5 * ref_var.max()
+    plan.destroy()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ a4 matching (stage-isolated)
 def _check_match(ex, ref):
     agree = ex["best_dst"] == ref["best_dst"]
