@@ -96,6 +96,21 @@ def test_var_map_and_partition(lib, wl):
     ctx.close()
 
 
+@pytest.mark.parametrize("patch,grid_h,grid_w", [(8, 9, 7), (16, 5, 6), (30, 3, 4), (1, 6, 33)])
+def test_grad_map_other_patch_sizes(lib, patch, grid_h, grid_w):
+    """Patch sizes other than 14: three patches per strip, one per strip, the largest accepted size and
+    single-pixel patches (the Grad map is then the Sobel magnitude itself)."""
+    g = torch.Generator().manual_seed(100 + patch)
+    img = torch.rand(3, 3, grid_h * patch, grid_w * patch, generator=g)
+    ctx = lib.LiteVGGT(3, grid_h, grid_w, 0.5, patch_px=patch)
+    got = ctx.grad_map(img.cuda())
+    ctx.poll()
+    ref = O.grad_map(img.numpy(), patch_px=patch)
+    assert got.shape == ref.shape
+    assert np.abs(to_f64(got) - ref).max() <= 1e-5 * max(ref.max(), 1e-3)
+    ctx.close()
+
+
 def test_scoring_maps_on_the_widest_grid(lib):
     """Grid of 33 x 64 patches: the widest row the library accepts (the Var map's per-row results and
     the Grad map's strips reach their limits), more than one block of 30 grid rows, and a frame whose
