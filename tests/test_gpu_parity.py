@@ -531,6 +531,14 @@ def test_abi_misuse_returns_error_codes(lib):
     _, tok = _inputs(wl)
     ctx = _ctx(lib, wl)
     other = lib.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, 0.25)
+    # shapes the kernels are not laid out for are refused when the context is made
+    for bad in (dict(patch_px=31), dict(grid_w=65)):
+        kw = dict(frames=wl.frames, grid_h=wl.grid_h, grid_w=wl.grid_w)
+        over = {k: v for k, v in bad.items() if k not in kw}
+        kw.update({k: v for k, v in bad.items() if k in kw})
+        with pytest.raises(lib.LiteVGGTError) as e:
+            lib.LiteVGGT(kw["frames"], kw["grid_h"], kw["grid_w"], 0.5, **over)
+        assert e.value.code == 2
     x = tok.cuda()
     _, ref = _oracle_plan(wl)
     plan = ctx.plan_import(ref["dst_of"])
