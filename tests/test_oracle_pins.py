@@ -90,7 +90,10 @@ def test_grad_against_library_convolution():
     k = torch.stack([kx, kx.t()]).unsqueeze(1)
     d = F.conv2d(F.pad(grey, (1, 1, 1, 1), mode="replicate"), k)
     ref = F.avg_pool2d(d.pow(2).sum(1, keepdim=True).sqrt(), 14)[:, 0].numpy()
-    np.testing.assert_allclose(O.grad_map(img), ref, rtol=1e-12, atol=1e-14)
+    # the library's float64 convolution sums in an order that depends on its thread split, and the
+    # square root magnifies a 1e-16 difference in gx, gy to about 1e-12 on a pixel whose gradient is
+    # near 1e-4; a wrong tap, sign or padding moves the result by O(1)
+    np.testing.assert_allclose(O.grad_map(img), ref, rtol=1e-10, atol=1e-12)
 
 
 def test_grad_brute_force_tiny():
