@@ -296,6 +296,7 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   size_t ml_off = 0;
   const size_t state_bytes = attention_state_bytes(z.n_merged, z.dim, z.heads, &ml_off);
   const size_t o_state = c.take<uint8_t>((long long)state_bytes);
+  const size_t o_kmax = c.take<float>((long long)z.frames * z.heads);
   const size_t o_status = c.take<uint32_t>(4);
   Workspace& ws = ctx->ws;
   if (cudaMalloc(&ws.base, c.off) != cudaSuccess) {
@@ -324,6 +325,7 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
     ws.attn_o_state = reinterpret_cast<float*>(ws.base + o_state);
     ws.attn_ml_state = reinterpret_cast<float*>(ws.base + o_state + ml_off);
   }
+  ws.attn_kmax = reinterpret_cast<float*>(ws.base + o_kmax);
   ws.status = reinterpret_cast<uint32_t*>(ws.base + o_status);
   if (cudaMemset(ws.base + o_var, 0, o_src - o_var) != cudaSuccess ||
       cudaMemset(ws.status, 0, 16) != cudaSuccess) {

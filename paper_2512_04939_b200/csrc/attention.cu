@@ -16,9 +16,11 @@
 //               thread cannot feed both tiles)
 //   warp  19    idle
 // Tensor memory (512 columns allocated, 480 used):
-//   [0,256)    S/P: tile t, half h at column t*128 + h*64.  S_th is 128 x 64 fp32; after the
-//              softmax threads have read it they overwrite its first 32 columns with P_th
-//              (bf16 pairs), which the second MMA reads as its A operand from there.
+//   [0,256)    S/P: tile t, half h at column t*128 + h*64.  S_th is 128 x 64 fp32.  A softmax
+//              thread reads its 32 columns and writes its 32 probabilities (16 columns of bf16
+//              pairs) over the start of the same 32 columns, so P_th sits in columns [0,16) and
+//              [32,48) of the half and no thread writes where another one reads; the second MMA
+//              takes its A operand from there, 8 columns (16 keys) per instruction.
 //   [256,416)  O_0, O_1 (fp32, 80 columns each: 64 output channels, then the row sum - the second
 //              MMA's B operand carries a column of ones next to V, so the tensor core adds up
 //              exactly the bf16 probabilities that it multiplies with V - and 15 unused columns)
@@ -33,13 +35,14 @@
 // needs a transpose.
 //
 // Softmax arithmetic.  At head dim 64 every score costs 256 tensor flops and one
-// exponential, and the special-function unit issues only 16 ex2 per clock per SM, half of
-// what the tensor cores would need.  A fixed share of the exponentials of every row can be
+// exponential, and the special-function unit issues only 16 ex2 per clock per SM (the packed
+// bf16x2 / f16x2 forms issue at half the rate, so they give the same 16 results per clock), half of
+// what the tensor cores would need.  A fixed share of the exponentials of every row is therefore
 // evaluated on the FMA pipes instead: round-to-nearest split x = n + f, |f| <= 1/2, a cubic
 // for 2^f (relative error 7.5e-5, far below the bf16 rounding of P) and n added into the
-// exponent field.  The share is a build-time constant and defaults to zero: on this part packed
-// fp32 instructions issue every second clock, so the cubic costs the FMA pipe about what ex2 costs
-// the special-function unit, and every share tried measured slower than none.
+// exponent field.  The share is a build-time constant, kFaPolyPairs of the 16 pairs of scores a
+// thread handles per step; 6 measured best (4 warps per scheduler on register data alone: 182
+// clocks per 32 scores against 257 with the special-function unit only; 8 pairs: 220).
 // Shared memory: K ring, V ring, and behind the V ring a block of the same size that holds the
 // ones column of the P V operand for every ring position (see the kernel).
 //
@@ -47,15 +50,28 @@
 // working set is the head's whole K/V; beyond about a quarter of the L2 that no longer stays
 // resident and every CTA would pull its tiles from HBM (measured: 2.4 TB per launch at 520 K
 // keys).  Long sequences are therefore swept in chunks of at most kFaChunkTiles key tiles, one
-// launch per chunk: a chunk's K/V of one head (32 MiB) stays in L2 while all query blocks pass
-// over it.  Between launches the un-normalised fp32 output rows, the reference maximum and the
-// row sum are parked in global memory (a few GB of traffic per launch instead).
+// launch per chunk: a chunk's K/V of one head (16 MiB) stays in L2 while all query blocks pass
+// over it.  Every launch starts its accumulators from zero and, at its end, adds its partial
+// output rows, row sums and reference to what the earlier chunks left in global memory (fp32,
+// round to nearest; a few GB of traffic per launch).  That also bounds the chain of additions
+// into one tensor-memory accumulator: carried through all 4067 key tiles of a 520 K-key sweep,
+// the accumulator picked up an error that grew in proportion to the number of keys (2.9e-3 of
+// the output's RMS at 252 K keys, 5.0e-3 at 520 K, against 2e-4 at 1.5 K).
 //
-// Online softmax in base 2 with a lazily updated reference maximum: the running output
-// is rescaled only when a row maximum grows by more than 2^8 over the reference (the
-// threads then first wait until the tile's last P V has retired), and the final division
-// by the row sum removes the reference again, so the result equals the plain softmax up
-// to rounding.
+// Softmax reference.  Any per-row constant m may be subtracted from the scores before the
+// exponential: the division by the row sum removes it again.  It only has to keep 2^(s - m)
+// inside the range of bf16 / fp32, it does not have to be the row maximum.  By Cauchy-Schwarz
+// every score of a row is at most B = |q| max_k |k| (times the softmax scale, in base-2 units), so
+// with m = B all exponents lie in [-2B, 0]; while 2B stays well inside the exponent range of
+// fp32 nothing underflows, every probability keeps its 8 significant bits and the fp32
+// accumulators their 24.  A small pass over K finds max_k |k|^2 per head before the sweep, each
+// softmax thread takes |q|^2 of its row while loading Q, and a warp pair whose rows all have
+// B <= kFaFixedRefLimit runs the sweep with that constant: no row maximum, no exchange between
+// the two threads of a row, no rescaling.  Rows with larger B (scores that could span more than
+// the exponent range allows) take the online form: base-2 softmax with a lazily updated reference
+// maximum, the running output rescaled only when a row maximum grows by more than 2^8 over the
+// reference (the threads then first wait until the tile's last P V has retired).  Both forms equal
+// the plain softmax up to rounding.
 #include "common.cuh"
 #include "runtime.h"
 
@@ -68,15 +84,22 @@ constexpr int kFaTileBytes = 128 * 64 * 2;
 constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 416;
 constexpr uint32_t kFaOCols = 80;  // 64 output channels, the row sum, 15 unused columns
 constexpr float kFaRescaleThreshold = 8.0f;
+// Largest Cauchy-Schwarz bound on the base-2 scores of a row for which the fixed reference is
+// used: probabilities go down to 2^-96, their products with |v| >= 2^-20 stay normal in fp32.
+#ifndef LV_FA_FIXED_REF_LIMIT
+#define LV_FA_FIXED_REF_LIMIT 48.0f
+#endif
+constexpr float kFaFixedRefLimit = LV_FA_FIXED_REF_LIMIT;
 #ifndef LV_FA_CHUNK_TILES
-#define LV_FA_CHUNK_TILES 1024
+#define LV_FA_CHUNK_TILES 512
 #endif
-constexpr int kFaChunkTiles = LV_FA_CHUNK_TILES;  // 131072 keys: K and V of one head = 32 MiB
-// Of every 8 consecutive pairs of scores, this many take the polynomial exponential.
+constexpr int kFaChunkTiles = LV_FA_CHUNK_TILES;  // 65536 keys: K and V of one head = 16 MiB
+// Of the 16 pairs of scores a thread handles per step, this many take the polynomial exponential
+// (fixed-reference form only, where every argument lies in [-2 * kFaFixedRefLimit, 0]).
 #ifndef LV_FA_POLY_PAIRS
-#define LV_FA_POLY_PAIRS 0
+#define LV_FA_POLY_PAIRS 6
 #endif
-constexpr int kFaPolyPairsPer8 = LV_FA_POLY_PAIRS;
+constexpr int kFaPolyPairs = LV_FA_POLY_PAIRS;
 
 struct FaBarriers {
   uint64_t q_ready;
@@ -101,11 +124,8 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 // 2^x for a pair of arguments on the FMA pipes.  Adding 1.5 * 2^23 rounds x to the nearest
 // integer n in the low mantissa bits; 2^(x - n) comes from a cubic fitted on [-1/2, 1/2] and
-// n is added to the exponent field.  Arguments are clamped at -120 (2^-120 stands in for
-// zero); the callers keep them below 2^8.
+// n is added to the exponent field.  Valid for arguments in [-120, 120].
 __device__ __forceinline__ float2 poly_exp2_pair(float2 x) {
-  x.x = fmaxf(x.x, -120.0f);
-  x.y = fmaxf(x.y, -120.0f);
   const float2 magic = make_float2(12582912.0f, 12582912.0f);
   const float2 t = __fadd2_rn(x, magic);
   const float2 n = __fadd2_rn(t, make_float2(-12582912.0f, -12582912.0f));
@@ -135,14 +155,17 @@ __device__ __forceinline__ void drain_ring(uint64_t* full, uint32_t issued, uint
 }
 
 // Exponentials of 32 scores of a row: p = 2^(s * scale - m_ref), packed to bf16 pairs (the row sum
-// is formed by the tensor core from these rounded values).
+// is formed by the tensor core from these rounded values).  The first kPoly of the 16 pairs take the
+// polynomial on the FMA pipes (callers guarantee arguments above -120 for them), the others the
+// special-function unit.
+template <int kPoly>
 __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 scale2, float2 neg_m2,
                                               uint32_t (&packed)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])), scale2, neg_m2);
     float2 p;
-    if ((i & 7) < kFaPolyPairsPer8) {
+    if (i < kPoly) {
       p = poly_exp2_pair(x);
     } else {
       p.x = fast_exp2(x.x);
@@ -161,7 +184,8 @@ template <bool kFirst, bool kLast>
 __global__ void __launch_bounds__(kFaThreads, 1)
 flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_state, float* __restrict__ ml_state,
-                       int seq_len, int dim, int tile_begin, int tile_end, float scale_log2e, uint32_t* status) {
+                       const float* __restrict__ k_norm2_max, int seq_len, int dim, int tile_begin, int tile_end,
+                       float scale_log2e, uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_k = smem;
@@ -285,14 +309,15 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           if (!mbar_wait(&bars->p_ready[t][h], j & 1, ctl)) { ok = false; break; }
           tc_fence_after();
           // 64 keys of V_j (64 rows of 128 bytes = 8192 bytes per half), 16 keys per instruction:
-          // 8 TMEM columns of P, 2048 bytes of V
+          // 8 TMEM columns of P (keys 0-31 in columns [0,16) of the half, keys 32-63 in [32,48)),
+          // 2048 bytes of V
           // second 64-column block of B = the ones block, one V ring further on
           const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192),
                                                   kFaStages * kFaTileBytes, 1024);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_ts(o_col, s_col + h * 64 + k * 8, v_desc + 128 * k, idesc_pv,
-                    (!first_chunk || (j | h | k) != 0) ? 1u : 0u);
+            umma_ts(o_col, s_col + h * 64 + (k >> 1) * 32 + (k & 1) * 8, v_desc + 128 * k, idesc_pv,
+                    (j | h | k) != 0 ? 1u : 0u);  // every launch starts its accumulators from zero
           if (last) {
             // no further Q K^T follows whose completion would tell the softmax threads that this
             // P V has retired
@@ -330,55 +355,72 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     const uint32_t s_addr = tmem_base + lane_base + kFaColS + t * 128;
     const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + c * 32;
     const uint32_t l_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + 64;  // row sum column (+15 unused)
+    float q_norm2 = 0.0f;  // |q|^2 of the whole row, summed in the same order by both of its threads
     {
       // this thread's half (32 channels) of its query row goes to tensor memory as it is
       uint32_t qreg[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) qreg[i] = 0u;
       if (row_live) {
-        const uint4* src = reinterpret_cast<const uint4*>(qkv + (size_t)row * 3 * dim + head * 64 + c * 32);
+        const uint4* src = reinterpret_cast<const uint4*>(qkv + (size_t)row * 3 * dim + head * 64);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const uint4 v = __ldg(src + i);
-          qreg[4 * i] = v.x; qreg[4 * i + 1] = v.y; qreg[4 * i + 2] = v.z; qreg[4 * i + 3] = v.w;
-        }
-      } else {
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int i = 0; i < 16; ++i) qreg[i] = 0u;
+          for (int e = 0; e < 4; ++e) {
+            q_norm2 = fmaf(bf16_lo(w[e]), bf16_lo(w[e]), q_norm2);
+            q_norm2 = fmaf(bf16_hi(w[e]), bf16_hi(w[e]), q_norm2);
+          }
+          if ((i >> 2) == c) {
+            qreg[4 * (i & 3)] = v.x; qreg[4 * (i & 3) + 1] = v.y; qreg[4 * (i & 3) + 2] = v.z; qreg[4 * (i & 3) + 3] = v.w;
+          }
+        }
       }
       tmem_st16(tmem_base + lane_base + kFaColQ + t * 32 + c * 16, qreg);
-      if (!first_chunk) {
-        // take up this row's running output (this thread's 32 channels) where the last chunk left it
-        uint32_t acc[32];
-        if (row_live) {
-          const uint4* src = reinterpret_cast<const uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint4 v = src[i];
-            acc[4 * i] = v.x; acc[4 * i + 1] = v.y; acc[4 * i + 2] = v.z; acc[4 * i + 3] = v.w;
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) acc[i] = 0u;
-        }
-        tmem_st32(o_addr, acc);
-        if (c == 1) {
-          uint32_t sum[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) sum[i] = 0u;
-          if (row_live) sum[0] = __float_as_uint(ml_state[((size_t)row * (dim / 64) + head) * 4 + 1]);
-          tmem_st16(l_addr, sum);
-        }
-      }
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->q_ready);
     }
     const float2 scale2 = make_float2(scale_log2e, scale_log2e);
-    float m_ref = -INFINITY;  // reference maximum, in log2 units (score * scale * log2 e)
-    // per (row, head) the previous chunk parked the reference maximum and the row sum
-    if (!first_chunk) m_ref = ml_state[((size_t)(row_live ? row : 0) * (dim / 64) + head) * 4];
+    // Cauchy-Schwarz bound on this row's scores in base-2 units; both threads of a row hold the same
+    // value, and both warps of a pair vote over the same 32 rows, so they agree on the form they run
+    const float score_bound = sqrtf(q_norm2 * k_norm2_max[blockIdx.z * gridDim.y + head]) * scale_log2e;
+    const bool fixed_ref = __all_sync(0xffffffffu, score_bound <= kFaFixedRefLimit ? 1 : 0) != 0;
+    float m_ref = -INFINITY;  // reference, in log2 units (score * scale * log2 e)
     bool ok = true;
     int pair_syncs = 0;  // both warps of a pair must pass the same number of pair barriers
+    if (fixed_ref) {
+      // ---- fixed reference: every exponent lies in [-2 * score_bound, 0]
+      m_ref = score_bound;
+      const float2 neg_m2 = make_float2(-m_ref, -m_ref);
+      pair_syncs = n_steps;  // this form has no pair barriers
+      for (int n = 0; n < n_steps; ++n) {
+        const int j = n >> 1, h = n & 1;
+        if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t s[32];
+        tmem_ld32(s_addr + h * 64 + c * 32, s);
+        tmem_ld_wait();
+        const int valid = seq_len - (tile_begin * 2 + n) * 64 - c * 32;
+        uint32_t packed[16];
+        if (valid < 32) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (i >= valid) s[i] = 0xff800000u;  // -inf: probability 0 (the polynomial cannot take it)
+          softmax_chunk<0>(s, scale2, neg_m2, packed);
+        } else {
+          softmax_chunk<kFaPolyPairs>(s, scale2, neg_m2, packed);
+        }
+        tmem_st16(s_addr + h * 64 + c * 32, packed);  // over the start of the columns just read
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
+      }
+    } else {
+    // ---- online form
     for (int n = 0; n < n_steps; ++n) {
       const int j = n >> 1, h = n & 1;
       if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
@@ -402,13 +444,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
         mx[g] = fmaxf(mx[g], __uint_as_float(sc[7]));
       }
       const float mx_own = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
-      // swap with the thread that holds the other 32 scores of this row; this barrier also orders
-      // that thread's P store (into columns this thread has just read) after the read
+      // swap with the thread that holds the other 32 scores of this row
       xchg->row_max[n & 1][t][c][row_in_tile] = mx_own;
       pair_barrier(barrier_id);
       ++pair_syncs;
       const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
-      if (first_chunk && n == 0) {
+      if (n == 0) {
         m_ref = mx_scaled;
       } else {
         const bool grow = mx_scaled > m_ref + kFaRescaleThreshold;
@@ -442,12 +483,13 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       }
       const float2 neg_m2 = make_float2(-m_ref, -m_ref);
       uint32_t packed[16];
-      softmax_chunk(s, scale2, neg_m2, packed);
-      tmem_st16(s_addr + h * 64 + c * 16, packed);  // P_th lies over the first 32 columns of S_th
+      softmax_chunk<0>(s, scale2, neg_m2, packed);
+      tmem_st16(s_addr + h * 64 + c * 32, packed);  // over the start of the columns just read
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
+    }
     }
     // a warp that gave up early still meets its partner at every barrier the partner may be in
     for (; pair_syncs < n_steps; ++pair_syncs) pair_barrier(barrier_id);
@@ -458,8 +500,34 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       tmem_ld16(l_addr, sum);
       tmem_ld_wait();
       if (row_live) {
+        float row_sum = __uint_as_float(sum[0]);
+        // each of the row's two threads keeps its own copy of {reference, row sum} in the state
+        float* ml_mine = ml_state + ((size_t)row * (dim / 64) + head) * 4 + 2 * c;
+        if (!first_chunk) {
+          // add what the earlier chunks left for this row, in fp32 with round-to-nearest: partial
+          // output, row sum, and - online form - their reference (the fixed form's is the same in
+          // every launch, bit for bit)
+          const float m_old = ml_mine[0], l_old = ml_mine[1];
+          float a_old = 1.0f, a_new = 1.0f;
+          if (m_old != m_ref) {
+            const float m_tot = fmaxf(m_old, m_ref);
+            a_old = fast_exp2(m_old - m_tot);
+            a_new = fast_exp2(m_ref - m_tot);
+            m_ref = m_tot;
+          }
+          const uint4* src = reinterpret_cast<const uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 v = src[i];
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              acc[4 * i + e] = __float_as_uint(fmaf(__uint_as_float(acc[4 * i + e]), a_new, __uint_as_float(w[e]) * a_old));
+          }
+          row_sum = fmaf(row_sum, a_new, l_old * a_old);
+        }
         if (last_chunk) {
-          const float inv = 1.0f / __uint_as_float(sum[0]);
+          const float inv = 1.0f / row_sum;
           uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -471,15 +539,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
             dst[q] = w;
           }
         } else {
-          // park the running state for the next chunk's launch
+          // leave the sum over the chunks so far for the next launch
           uint4* dst = reinterpret_cast<uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i) dst[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
-          float* ml_row = ml_state + ((size_t)row * (dim / 64) + head) * 4;
-          if (c == 0) {
-            ml_row[0] = m_ref;
-            ml_row[1] = __uint_as_float(sum[0]);
-          }
+          ml_mine[0] = m_ref;
+          ml_mine[1] = row_sum;
         }
       }
     }
@@ -493,16 +558,62 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   }
 }
 
+// max_k |k|^2 per (sequence, head), for the Cauchy-Schwarz bound on a row's scores.  Warp per key
+// row: the 128 16-byte pieces of a K row go to the lanes in four passes, eight neighbouring lanes
+// share a head.  Non-negative floats order like their bit patterns, so the maximum is an integer
+// atomicMax on a zeroed array.
+constexpr int kKnormWarps = 8;
+__global__ void __launch_bounds__(kKnormWarps * 32)
+key_norm_max_kernel(const __nv_bfloat16* __restrict__ qkv, int seq_len, int dim, float* __restrict__ k_norm2_max) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int seq = blockIdx.y, heads = dim / 64;
+  float best[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  for (int r = blockIdx.x * kKnormWarps + warp; r < seq_len; r += gridDim.x * kKnormWarps) {
+    const uint4* src = reinterpret_cast<const uint4*>(qkv + ((size_t)seq * seq_len + r) * 3 * dim + dim);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint4 v = __ldg(src + lane + 32 * j);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      float sum = 0.0f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        sum = fmaf(bf16_lo(w[e]), bf16_lo(w[e]), sum);
+        sum = fmaf(bf16_hi(w[e]), bf16_hi(w[e]), sum);
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      best[j] = fmaxf(best[j], sum);
+    }
+  }
+  if ((lane & 7) == 0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      atomicMax(reinterpret_cast<unsigned int*>(k_norm2_max) + seq * heads + (lane >> 3) + 4 * j,
+                __float_as_uint(best[j]));
+  }
+}
+
 cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long seq_len, int n_seq,
                                    __nv_bfloat16* o, cudaStream_t s, int* launches) {
   if (seq_len == 0 || n_seq == 0) return cudaSuccess;
   const int dim = ctx->sz.dim;
+  if (dim != 1024 || ctx->ws.attn_kmax == nullptr) return cudaErrorInvalidValue;
+  {
+    cudaError_t e = cudaMemsetAsync(ctx->ws.attn_kmax, 0, (size_t)n_seq * ctx->sz.heads * sizeof(float), s);
+    if (e != cudaSuccess) return e;
+    long long blocks = (seq_len + 63) / 64;
+    if (blocks > 2048) blocks = 2048;
+    key_norm_max_kernel<<<dim3((unsigned)blocks, (unsigned)n_seq), kKnormWarps * 32, 0, s>>>(qkv, (int)seq_len, dim,
+                                                                                            ctx->ws.attn_kmax);
+    ++*launches;
+  }
   const long long rows = seq_len * n_seq;
   CUtensorMap tmap;
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap, qkv, (uint64_t)3 * dim, (uint64_t)rows, (uint64_t)3 * dim, 64, 128))
     return cudaErrorInvalidValue;
-  using Kernel = void (*)(const CUtensorMap, const __nv_bfloat16*, __nv_bfloat16*, float*, float*, int, int, int, int,
-                          float, uint32_t*);
+  using Kernel = void (*)(const CUtensorMap, const __nv_bfloat16*, __nv_bfloat16*, float*, float*, const float*, int,
+                          int, int, int, float, uint32_t*);
   const Kernel kernels[2][2] = {{flash_attention_kernel<false, false>, flash_attention_kernel<false, true>},
                                 {flash_attention_kernel<true, false>, flash_attention_kernel<true, true>}};
   for (int a = 0; a < 2; ++a)
@@ -522,15 +633,15 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   for (int begin = 0; begin < n_tiles; begin += per_chunk) {
     const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
     kernels[begin == 0][end == n_tiles]<<<grid, kFaThreads, kFaSmemBytes, s>>>(
-        tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, (int)seq_len, dim, begin, end, scale_log2e,
-        ctx->ws.status);
+        tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, ctx->ws.attn_kmax, (int)seq_len, dim, begin, end,
+        scale_log2e, ctx->ws.status);
     ++*launches;
   }
   return cudaGetLastError();
 }
 
-// Rows of fp32 running output and of {reference maximum, two partial row sums, pad} per head that the
-// chunked sweep parks between launches; zero when m fits one chunk.
+// Rows of fp32 partial output and of {reference, row sum} x 2 per head (one copy per thread of a row)
+// that the chunked sweep sums up between launches; zero when m fits one chunk.
 size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset) {
   const long long n_tiles = (m + 127) / 128;
   if (n_tiles <= kFaChunkTiles) {

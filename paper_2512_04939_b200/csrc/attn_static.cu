@@ -21,7 +21,8 @@ constexpr size_t kStatusBytes = 256;
 constexpr size_t kQkvBytes = (size_t)kStaticMaxRows * 3 * kStaticDim * 2;
 constexpr size_t kOBytes = (size_t)kStaticMaxRows * kStaticDim * 2;
 
-// [ status word, padded | qkv bf16 [1024, 3072] | o bf16 [1024, 1024] ]  = 8 MiB + 256 B
+// [ status word, 16 floats of per-head key norms at byte 64, padding | qkv bf16 [1024, 3072] |
+//   o bf16 [1024, 1024] ]  = 8 MiB + 256 B
 static __device__ __align__(256) unsigned char g_attn_scratch[kStatusBytes + kQkvBytes + kOBytes];
 
 constexpr int kMaxDevices = 64;
@@ -104,6 +105,7 @@ extern "C" litevggt_status litevggt_global_attn_static(const void* x_merged, int
   local.sz.dim = kStaticDim;
   local.sz.heads = kStaticHeads;
   local.ws.status = status;
+  local.ws.attn_kmax = reinterpret_cast<float*>(dev->scratch + 64);  // zeroed by the attention launcher
   int n = 0;
   cudaError_t e = lv::launch_linear(&local, static_cast<const __nv_bfloat16*>(x_merged), m, kStaticDim,
                                     static_cast<const __nv_bfloat16*>(w_qkv), 3 * kStaticDim,

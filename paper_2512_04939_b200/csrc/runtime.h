@@ -53,6 +53,7 @@ struct Workspace {
   __nv_bfloat16* attn_o = nullptr; // [M, D]
   float* attn_o_state = nullptr;   // [M, D] running output between key chunks (long sequences only)
   float* attn_ml_state = nullptr;  // [M, heads, 4] reference maximum and partial row sums
+  float* attn_kmax = nullptr;      // [max(frames, 1), heads] largest |k|^2 per sequence and head
   // whole-layer-from-host staging
   __nv_bfloat16* stage_x = nullptr;   // [N, D]
   __nv_bfloat16* stage_xm = nullptr;  // [M, D]

@@ -11,5 +11,6 @@ from .generate import (  # noqa: F401
     make_tokens,
     make_attention_weights,
     make_block_weights,
+    make_peaked_attention_inputs,
     make_workload_inputs,
 )

@@ -221,6 +221,36 @@ def make_attention_weights(wl: Workload, layer: int, device="cpu", dim: int = DI
     return w_qkv, b_qkv, w_o, b_o
 
 
+def make_peaked_attention_inputs(m: int, seed: int, device="cpu", groups: int = 4099, sharpness: float = 4.0,
+                                 dim: int = DIM):
+    """Rows and projection weights under which softmax attention is far from uniform.
+
+    Row j = base[j % groups] + 0.5 * noise_j with unit-variance base and noise, and the query
+    weights are ``sharpness`` times the key weights, so a query scores highest against itself and
+    next against the other rows of its own group, which lie ``groups`` rows apart through the whole
+    sequence (about m / groups of them, with different weights and different values).  Random-init
+    0.02 weights on the token generator's rows give nearly uniform attention, under which a lost or
+    repeated stretch of keys barely moves the output; these inputs make it move.
+    Returns (x [m, dim] bf16, w_qkv, b_qkv, w_o, b_o) like make_attention_weights."""
+    dev = torch.device(device)
+    g = _gen(seed, dev)
+    bf = torch.bfloat16
+    base = torch.randn(groups, dim, generator=g, device=dev)
+    x = torch.empty(m, dim, dtype=bf, device=dev)
+    chunk = 1 << 16
+    for r0 in range(0, m, chunk):
+        r1 = min(m, r0 + chunk)
+        idx = torch.arange(r0, r1, device=dev) % groups
+        x[r0:r1] = (base[idx] + 0.5 * torch.randn(r1 - r0, dim, generator=g, device=dev)).to(bf)
+    w_k = 0.02 * torch.randn(dim, dim, generator=g, device=dev)
+    w_v = 0.02 * torch.randn(dim, dim, generator=g, device=dev)
+    w_qkv = torch.cat([sharpness * w_k, w_k, w_v]).to(bf)
+    b_qkv = (0.02 * torch.randn(3 * dim, generator=g, device=dev)).to(bf)
+    w_o = (0.02 * torch.randn(dim, dim, generator=g, device=dev)).to(bf)
+    b_o = (0.02 * torch.randn(dim, generator=g, device=dev)).to(bf)
+    return x, w_qkv, b_qkv, w_o, b_o
+
+
 def make_block_weights(wl: Workload, layer: int, device="cpu", dim: int = DIM):
     """Weights of the other sub-layers of one aggregator block, bf16: two LayerNorms (gamma near 1,
     beta near 0), the frame-attention layer (as make_attention_weights) and the MLP of ratio 4

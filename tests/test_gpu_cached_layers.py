@@ -9,7 +9,7 @@ import torch
 
 import oracle as O
 from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
-from helpers import bf16_bound, rel_err, to_f64
+from helpers import LAYER_NOISE, bf16_bound, check_bf16, rel_err, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -54,16 +54,162 @@ def test_plan_cached_across_four_layers_c2():
         # oracle on this layer's GPU input with the cached indices (sampled outputs)
         x64 = to_f64(x)
         ref_m = O.merge(x64, ex["dst_of"], m)
-        assert rel_err(to_f64(xm), ref_m) <= bf16_bound(ref_m), f"merge, layer {layer}"
+        check_bf16(f"C2 layer {layer}: merge with the cached plan", to_f64(xm), ref_m)
         w64 = [to_f64(t) for t in w]
         ref_y = O.global_attention(to_f64(xm), *w64, heads=16, rows=rows)
-        assert rel_err(to_f64(ym)[rows], ref_y) <= 2 * bf16_bound(ref_y), f"attention, layer {layer}"
+        check_bf16(f"C2 layer {layer}: attention layer", to_f64(ym)[rows], ref_y, noise=LAYER_NOISE, sampled=True)
         ref_out = O.unmerge(to_f64(ym), ex["dst_of"], x64)[toks]
-        assert rel_err(to_f64(out)[toks], ref_out) <= bf16_bound(ref_out), f"unmerge, layer {layer}"
+        check_bf16(f"C2 layer {layer}: unmerge with residual", to_f64(out)[toks], ref_out, sampled=True)
         # conservation of the size-weighted sum under the cached plan on drifting features
         lhs = (ex["size"][:, None] * ref_m).sum(0)
         np.testing.assert_allclose(lhs, x64.sum(0), rtol=0, atol=1e-6 * np.abs(x64).sum(0).max())
         x = out
     assert builds == 1  # four layers, interval 6: computed once, reused three times
+    plan.destroy()
+    ctx.close()
+
+
+def _check_plan_against_oracle(tag, ctx, plan, x, grad64, wl, interval_layer):
+    """A plan built by the library (first build or refresh in place) against the oracle on the very
+    features the GPU used: classes equal except at score near-ties (>= 99.9 % overall), matching
+    judged on the GPU's own classes (exact where the oracle's margin exceeds 1e-3, >= 99.9 % overall,
+    similarities within 1e-5), selection and index arrays bit-exact given the GPU's matches."""
+    from helpers import report
+
+    ex = ctx.plan_export(plan)
+    x64 = to_f64(x)
+    ref = O.merge_plan(x64, grad64, wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio)
+    diff = np.flatnonzero(ex["cls"] != ref["cls"])
+    assert diff.size <= 1e-3 * ex["cls"].size, f"{tag}: {diff.size} tokens in another class"
+    ga = ref["ga"].reshape(wl.frames, -1)
+    for i in diff:
+        f, t = divmod(int(i), wl.tokens_per_frame)
+        others = np.delete(ga[f], t - 5)
+        assert np.abs(others - ga[f, t - 5]).min() < 1e-5, f"{tag}: class differs without a near-tie"
+    src_idx = np.flatnonzero(ex["cls"] == O.CLS_SRC)
+    dst_idx = np.flatnonzero(ex["cls"] == O.CLS_DST)
+    if diff.size == 0:
+        best, sim1, sim2 = ref["best_dst"], ref["best_sim"], ref["second_sim"]
+    else:
+        best, sim1, sim2 = O.match(x64, src_idx, dst_idx)
+    margin = sim1 - sim2
+    agree = ex["best_dst"] == best
+    report(f"{tag}: plan at layer {interval_layer}", class_differences=int(diff.size), match_agreement=float(agree.mean()),
+           near_ties_accepted=int((~agree).sum()), margin_below_1e_3=float((margin < 1e-3).mean()),
+           margin_below_1e_4=float((margin < 1e-4).mean()), margin_below_1e_5=float((margin < 1e-5).mean()))
+    assert np.all(agree[margin > 1e-3]), f"{tag}: argmax differs although the oracle's margin exceeds 1e-3"
+    # 99.9 % agreement; on a population of a few hundred rows (config C1 has 501 src tokens) that is
+    # less than one row, so one near-tie (similarity within 1e-5 of the oracle's best, below) may differ
+    assert (~agree).sum() <= max(1, int(1e-3 * agree.size)), f"{tag}: {(~agree).sum()} of {agree.size} matches differ"
+    assert np.abs(ex["best_sim"] - sim1).max() <= 1e-5, tag
+    n_remove = O.derived_sizes(wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio)["R"]
+    dst_of, size, kept = O.select_and_index(ex["cls"], ex["best_dst"], ex["best_sim"], n_remove)
+    assert np.array_equal(ex["dst_of"], dst_of) and np.array_equal(ex["size"], size), tag
+    assert np.array_equal(ex["kept_idx"], kept), tag
+    return ex
+
+
+def test_plan_refreshed_in_place_on_drifted_features_c4_schedule():
+    """Config C4's schedule on C4's grid and merge ratio (every src token merged), 32 frames instead
+    of 500 so that the oracle can rebuild the whole plan: 8 global layers, the plan built at layer 0,
+    reused by layers 1-5, rebuilt IN PLACE at layer 6 on the features the residual stream has drifted
+    to, reused by layer 7 (Sec. 3.4: indices recomputed every 6 layers).  Both builds are compared
+    with the oracle's plan on the GPU's own input of that layer; every layer's merge, attention and
+    unmerge with the oracle applied to the cached indices."""
+    import dataclasses
+
+    import paper_2512_04939_b200 as pkg
+
+    wl = dataclasses.replace(WORKLOADS["C4"], name="C4x32", frames=32, global_layers=8)
+    images = make_images(wl)
+    tokens = make_tokens(wl, images)
+    grad64 = O.grad_map(images.numpy())
+    ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, recompute_interval=6)
+    assert ctx.n_merged == ctx.n_tokens - ctx.n_src  # saturated: the paper's rule
+    x = tokens.cuda()
+    grad = ctx.grad_map(images.cuda())
+    rng = np.random.default_rng(23)
+    m = ctx.n_merged
+    rows = np.unique(np.concatenate([rng.choice(m, 40, replace=False), [0, m - 1]]))
+    toks = np.unique(np.concatenate([rng.choice(ctx.n_tokens, 200, replace=False), [0, ctx.n_tokens - 1]]))
+    plan, builds, ex, first = None, 0, None, None
+    for layer in range(wl.global_layers):
+        assert bool(ctx.should_refresh(plan, layer)) == (plan is None or O.should_refresh(layer, 6))
+        if ctx.should_refresh(plan, layer):
+            handle_before = None if plan is None else plan.handle.value
+            plan = ctx.merge_plan(x, grad, plan)
+            assert handle_before is None or plan.handle.value == handle_before  # same object, rebuilt in place
+            builds += 1
+            ctx.poll()
+            ex = _check_plan_against_oracle("C4x32", ctx, plan, x, grad64, wl, layer)
+            if first is None:
+                first = ex
+            else:
+                # the features have drifted: the refreshed plan is a different one
+                assert (ex["dst_of"] != first["dst_of"]).mean() > 0.01
+        w = [t.cuda() for t in make_attention_weights(wl, layer)]
+        xm = ctx.merge(plan, x)
+        ym = ctx.global_attn(xm, *w)
+        out = ctx.unmerge(plan, ym, x)
+        ctx.poll()
+        x64 = to_f64(x)
+        ref_m = O.merge(x64, ex["dst_of"], m)
+        check_bf16(f"C4x32 layer {layer}: merge with the cached plan", to_f64(xm), ref_m)
+        ref_y = O.global_attention(to_f64(xm), *[to_f64(t) for t in w], heads=16, rows=rows)
+        check_bf16(f"C4x32 layer {layer}: attention layer", to_f64(ym)[rows], ref_y, noise=LAYER_NOISE, sampled=True)
+        ref_out = O.unmerge(to_f64(ym), ex["dst_of"], x64)[toks]
+        check_bf16(f"C4x32 layer {layer}: unmerge with residual", to_f64(out)[toks], ref_out, sampled=True)
+        x = out
+    assert builds == 2
+    plan.destroy()
+    ctx.close()
+
+
+def _golden_schedule():
+    import os
+
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "recompute_schedule.txt")
+    return {int(a): int(b) for a, b in (ln.split() for ln in open(path) if ln[0] != "#")}
+
+
+@pytest.mark.parametrize("interval", [1, 2, 3, 6, 24])
+def test_recompute_intervals_of_the_caching_ablation(interval):
+    """The recompute intervals of the paper's supplementary "Caching merge indices" table over 24
+    global layers (config C1's sequence, so that the oracle can rebuild every plan): the library's
+    refresh decision equals the oracle's at every layer, the number of plan builds equals the
+    paper's count, and every refreshed plan equals the oracle's on the drifted features of that
+    layer.  The last layer's output is checked with the cached indices."""
+    import paper_2512_04939_b200 as pkg
+
+    wl = WORKLOADS["C1"]
+    images = make_images(wl)
+    tokens = make_tokens(wl, images)
+    grad64 = O.grad_map(images.numpy())
+    ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, recompute_interval=interval)
+    x = tokens.cuda()
+    grad = ctx.grad_map(images.cuda())
+    plan, builds, ex = None, 0, None
+    for layer in range(24):
+        want = O.should_refresh(layer, interval)
+        assert bool(ctx.should_refresh(plan, layer)) == bool(want or plan is None)
+        if ctx.should_refresh(plan, layer):
+            plan = ctx.merge_plan(x, grad, plan)
+            builds += 1
+            ctx.poll()
+            ex = _check_plan_against_oracle(f"C1 interval {interval}", ctx, plan, x, grad64, wl, layer)
+        w = [t.cuda() for t in make_attention_weights(wl, layer)]
+        xm = ctx.merge(plan, x)
+        ym = ctx.global_attn(xm, *w)
+        out = ctx.unmerge(plan, ym, x)
+        ctx.poll()
+        if layer == 23:
+            x64 = to_f64(x)
+            ref_y = O.global_attention(O.merge(x64, ex["dst_of"], ctx.n_merged), *[to_f64(t) for t in w], heads=16)
+            # the attention branch (stored bf16 intermediates, none in the oracle) is about half of the
+            # output's RMS at this depth
+            check_bf16(f"C1 interval {interval}: layer 23 with the cached plan", to_f64(out),
+                       O.unmerge(ref_y, ex["dst_of"], x64), noise=LAYER_NOISE / 2)
+        x = out
+    assert builds == _golden_schedule()[interval]
     plan.destroy()
     ctx.close()

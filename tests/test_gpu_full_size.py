@@ -9,8 +9,9 @@ import pytest
 import torch
 
 import oracle as O
-from synthdata import WORKLOADS, make_attention_weights, make_block_weights, make_images, make_tokens
-from helpers import bf16_bound, rel_err, to_f64
+from synthdata import (WORKLOADS, make_attention_weights, make_block_weights, make_images,
+                       make_peaked_attention_inputs, make_tokens)
+from helpers import CORE_NOISE, LAYER_NOISE, bf16_bound, check_bf16, rel_err, report, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -97,23 +98,36 @@ def test_partition_counts_everywhere_and_classes_on_sampled_frames(run):
         assert diff.size <= 4
 
 
+N_MATCH_ROWS = 4096
+
+
 def test_matches_on_sampled_src_rows(run):
-    ex, tokens = run["ex"], run["tokens"]
+    """4096 seeded src rows against every anchor of the sequence (the oracle's match on a compact
+    copy: anchors first, then the sampled rows).  The stated tolerance in full: the argmax equals the
+    oracle's wherever the oracle's top-1 / top-2 margin exceeds 1e-3, at least 99.9 % of the rows agree,
+    and a row that differs is a near-tie (its similarity within 1e-5 of the oracle's best).  The margin
+    histogram and the agreement are reported with the result."""
+    ex, tokens, wl = run["ex"], run["tokens"], run["wl"]
     src_idx = np.flatnonzero(ex["cls"] == O.CLS_SRC)
     dst_idx = np.flatnonzero(ex["cls"] == O.CLS_DST)
     rng = np.random.default_rng(5)
-    rows = np.sort(rng.choice(src_idx.size, 48, replace=False))
-    # compact copy: anchors first, then the sampled src rows
+    rows = np.sort(rng.choice(src_idx.size, min(N_MATCH_ROWS, src_idx.size), replace=False))
     xd = to_f64(tokens[torch.from_numpy(dst_idx).cuda()])
     xs = to_f64(tokens[torch.from_numpy(src_idx[rows]).cuda()])
     x_small = np.concatenate([xd, xs])
-    best, sim1, sim2 = O.match(x_small, dst_idx.size + np.arange(rows.size), np.arange(dst_idx.size))
+    del xd, xs
+    best, sim1, sim2 = O.match(x_small, dst_idx.size + np.arange(rows.size), np.arange(dst_idx.size), chunk=512)
     best_token = dst_idx[best]
     margin = sim1 - sim2
     agree = ex["best_dst"][rows] == best_token
+    report(f"{wl.name}: matching on {rows.size} sampled src rows x {dst_idx.size} anchors",
+           agreement=float(agree.mean()), near_ties_accepted=int((~agree).sum()),
+           margin_below_1e_5=float((margin < 1e-5).mean()), margin_below_1e_4=float((margin < 1e-4).mean()),
+           margin_below_1e_3=float((margin < 1e-3).mean()), margin_median=float(np.median(margin)),
+           best_sim_max_abs_diff=float(np.abs(ex["best_sim"][rows] - sim1).max()))
     assert np.all(agree[margin > 1e-3]), "argmax differs although the oracle's margin exceeds 1e-3"
     assert np.abs(ex["best_sim"][rows] - sim1).max() <= 1e-5
-    assert agree.mean() >= 0.9  # the full-population bound (99.9 %) is checked at the small sizes
+    assert agree.mean() >= 0.999
 
 
 def test_selection_and_index_arrays_bit_exact_given_the_matches(run):
@@ -159,10 +173,10 @@ def test_attention_layer_on_sampled_rows(run):
     o_gpu = ctx.debug_buffer(1)
     # projections on the sampled rows
     ref_qkv = O.linear(to_f64(xm[rows_t]), w_qkv, b_qkv)
-    assert rel_err(to_f64(qkv_gpu[rows_t]), ref_qkv) <= bf16_bound(ref_qkv), "qkv projection"
+    check_bf16(f"{run['wl'].name}: qkv projection", to_f64(qkv_gpu[rows_t]), ref_qkv, sampled=True)
     o_rows = to_f64(o_gpu[rows_t])
     ref_y = O.linear(o_rows, w_o, b_o)
-    assert rel_err(to_f64(run["ym"][rows_t]), ref_y) <= bf16_bound(ref_y), "output projection"
+    check_bf16(f"{run['wl'].name}: output projection", to_f64(run["ym"][rows_t]), ref_y, sampled=True)
     # attention core: the sampled queries against all M keys, three heads, one head at a time
     # (the oracle is called with heads=1 on that head's [Q | K | V] columns)
     for head in (0, 6, 15):
@@ -171,14 +185,69 @@ def test_attention_layer_on_sampled_rows(run):
         k = to_f64(qkv_gpu[:, 1024 + cols])
         v = to_f64(qkv_gpu[:, 2048 + cols])
         ref_o = O.attention_core(np.concatenate([q, k, v], axis=1), heads=1, rows=rows)
-        weighted_abs = O.attention_core(np.concatenate([q, k, np.abs(v)], axis=1), heads=1, rows=rows)
-        rms = float(np.sqrt(np.mean(ref_o * ref_o)))
-        # Output rounding + bf16 probabilities (2^-8 * sum p|v| / sum p), as in the small-size test.
-        # With so few sampled outputs the rounding term is the worst case for their magnitudes
-        # (half a bf16 ulp) rather than the rounding error the reference values happen to have.
-        half_ulp = float((2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref_o), 1e-30))) - 8)).max()) / rms
-        bound = max(1e-2, half_ulp + 2e-3) + 2.0 ** -8 * float(weighted_abs.max()) / rms
-        assert rel_err(o_rows[:, 64 * head:64 * head + 64], ref_o) <= bound, f"attention core, head {head}"
+        check_bf16(f"{run['wl'].name}: attention core, stock weights, head {head}", o_rows[:, 64 * head:64 * head + 64],
+                   ref_o, sampled=True, elem_noise=CORE_NOISE)
+
+
+def key_chunk_edges(m):
+    """First key row of every key chunk but the first, as the attention launcher splits a long
+    sequence: tiles of 128 keys, balanced chunks of at most 512 tiles."""
+    n_tiles = -(-m // 128)
+    n_chunks = -(-n_tiles // 512)
+    per_chunk = -(-n_tiles // n_chunks)
+    return [c * per_chunk * 128 for c in range(1, n_chunks)], per_chunk * 128
+
+
+@pytest.mark.parametrize("name", ["C3", "C4", "C5"])
+def test_attention_core_with_peaked_softmax_across_key_chunks(name):
+    """The attention core at the merged lengths of C3, C4 and C5 on inputs whose softmax is far from
+    uniform: every query's mass sits on itself and on the ~M/4099 rows of its group, which lie 4099
+    rows apart through the whole sequence, so every key chunk (C3: 2, C4: 4, C5: 8) carries a share of every
+    output.  Sampled queries sit on both sides of every chunk boundary, at tile edges and at random.
+    A chunk left out on the oracle's side must move the result far beyond the tolerance."""
+    import paper_2512_04939_b200 as pkg
+
+    wl = WORKLOADS[name]
+    ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio)
+    m = ctx.n_merged
+    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, wl.seed + 9, "cuda")
+    ctx.global_attn(x, w_qkv, b_qkv, w_o, b_o)
+    ctx.poll()
+    edges, chunk_rows = key_chunk_edges(m)
+    rng = np.random.default_rng(17)
+    rows = [0, 127, 128, 255, 256, m - 129, m - 128, m - 1] + list(rng.choice(m, 16, replace=False))
+    for e in edges:
+        rows += [e - 129, e - 128, e - 1, e, e + 127, e + 128]
+    rows = np.unique(np.asarray(rows, dtype=np.int64))
+    rows_t = torch.from_numpy(rows).cuda()
+    qkv_gpu, o_gpu = ctx.debug_buffer(0), ctx.debug_buffer(1)
+    o_rows = to_f64(o_gpu[rows_t])
+    for head in (0, 9, 15):
+        cols = torch.arange(64, device="cuda") + 64 * head
+        qkv_h = np.concatenate([to_f64(qkv_gpu[:, cols]), to_f64(qkv_gpu[:, 1024 + cols]),
+                                to_f64(qkv_gpu[:, 2048 + cols])], axis=1)
+        ref_o = O.attention_core(qkv_h, heads=1, rows=rows)
+        got = o_rows[:, 64 * head:64 * head + 64]
+        check_bf16(f"{name}: attention core, peaked softmax, head {head}", got, ref_o, sampled=True, elem_noise=CORE_NOISE)
+        bound = bf16_bound(ref_o)
+        # planted on the oracle's side: without the keys of chunk c (queries taken outside it)
+        for c in range(len(edges) + 1):
+            lo, hi = c * chunk_rows, min(m, (c + 1) * chunk_rows)
+            outside = (rows < lo) | (rows >= hi)
+            kept = np.concatenate([qkv_h[:lo], qkv_h[hi:]])
+            if kept.shape[0] == 0:
+                continue
+            moved = np.where(rows[outside] >= hi, rows[outside] - (hi - lo), rows[outside])
+            ref_short = O.attention_core(kept, heads=1, rows=moved)
+            lost = rel_err(got[outside], ref_short)
+            report(f"{name}: head {head}, oracle without key chunk {c}", err_over_rms=lost, bound=bound)
+            # a chunk holds 1/8 (C5) to 1/2 (C3) of every row's mass: several times the tolerance
+            assert lost > 5 * bound, f"dropping key chunk {c} on the oracle's side goes unnoticed"
+            del kept
+        del qkv_h
+    ctx.close()
+    del x
+    torch.cuda.empty_cache()
 
 
 def test_block_sublayers_on_sampled_rows_and_frames(run):

@@ -6,8 +6,9 @@ import pytest
 import torch
 
 import oracle as O
-from synthdata import WORKLOADS, Workload, make_attention_weights, make_block_weights, make_images, make_tokens
-from helpers import bf16_bound, rel_err, to_f64
+from synthdata import (WORKLOADS, Workload, make_attention_weights, make_block_weights, make_images,
+                       make_peaked_attention_inputs, make_tokens)
+from helpers import CORE_NOISE, LAYER_NOISE, bf16_bound, bf16_round, check_bf16, rel_err, report, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -274,7 +275,7 @@ def test_merge_unmerge_with_oracle_plan(lib, wl):
     x64 = to_f64(tok)
     ref_m = O.merge(x64, ref["dst_of"], ref["sizes"]["M"])
     got = to_f64(xm)
-    assert rel_err(got, ref_m) <= bf16_bound(ref_m)
+    check_bf16(f"{wl.name}: merge", got, ref_m)
     single = ref["size"] == 1
     assert np.array_equal(got[single], x64[ref["kept_idx"][single]])  # bit-exact copies
     # conservation of size-weighted sums, up to the one bf16 rounding per merged row
@@ -286,7 +287,7 @@ def test_merge_unmerge_with_oracle_plan(lib, wl):
     assert np.array_equal(to_f64(out), O.unmerge(to_f64(ym), ref["dst_of"]))
     out_r = ctx.unmerge(plan, ym, x)
     ref_r = O.unmerge(to_f64(ym), ref["dst_of"], x64)
-    assert rel_err(to_f64(out_r), ref_r) <= bf16_bound(ref_r)
+    check_bf16(f"{wl.name}: unmerge with residual", to_f64(out_r), ref_r)
     ctx.poll()
     plan.destroy()
     ctx.close()
@@ -305,24 +306,30 @@ def test_linear(lib, m, k, n):
         got = ctx.linear(a.cuda(), w.cuda(), None if bias is None else bias.cuda())
         ctx.poll()
         ref = to_f64(a) @ to_f64(w).T + (0 if bias is None else to_f64(bias))
-        assert rel_err(to_f64(got), ref) <= bf16_bound(ref)
+        check_bf16(f"linear {m}x{k}x{n}", to_f64(got), ref)
     ctx.close()
 
 
 # ------------------------------------------------------------------ a7-a9 attention
-def attention_core_bound(qkv, ref_o):
-    """Tolerance of the attention core in bf16 arithmetic.  Besides the rounding of the output
-    itself (bf16_bound), the probabilities enter the second tensor-core product as bf16, each
-    with a relative error of up to 2^-8 (half an ulp of an 8-bit significand, at the bottom of a
-    binade), which moves an output by at most 2^-8 * sum_i p_i |v_i| / sum_i p_i.  When attention is
-    nearly uniform all probabilities round the same way, so this is a bias, not noise.  When a few keys dominate a row the two terms are of
-    the same size, so the second one is part of the bound, evaluated with the oracle on |V|."""
-    d = qkv.shape[1] // 3
-    abs_v = qkv.copy()
-    abs_v[:, 2 * d:] = np.abs(abs_v[:, 2 * d:])
-    weighted_abs = O.attention_core(abs_v, heads=16)
-    rms = float(np.sqrt(np.mean(ref_o * ref_o)))
-    return bf16_bound(ref_o) + 2.0 ** -8 * float(weighted_abs.max()) / rms
+# Tolerances of the attention layer.  Each stage is judged on the GPU's own upstream result, so the
+# stated bound (1e-2 of the RMS, or the output's own rounding floor + 2e-3) applies as it is: the
+# core normalises with the sum of the very bf16 probabilities that multiply V, so their rounding
+# (relative 2^-9, independent from key to key) enters as noise of 2^-9 sqrt(sum p^2 (v-o)^2) / sum p,
+# far below the rounding of the output unless a single key holds the row - and then v = o.
+# End to end the oracle rounds nothing while the GPU stores qkv, o and y in bf16: helpers.LAYER_NOISE
+# is the allowance for that.
+
+
+def score_bounds(qkv, heads=16):
+    """Cauchy-Schwarz bound |q| max_k |k| / sqrt(dh) * log2(e) on the base-2 scores of every
+    (row, head): which of the kernel's two softmax forms a row takes depends on it."""
+    m, d = qkv.shape[0], qkv.shape[1] // 3
+    q = qkv[:, :d].reshape(m, heads, d // heads)
+    k = qkv[:, d:2 * d].reshape(m, heads, d // heads)
+    return np.sqrt((q * q).sum(-1)) * np.sqrt((k * k).sum(-1)).max(0) / np.sqrt(d // heads) * np.log2(np.e)
+
+
+FIXED_REF_LIMIT = 48.0  # the library's kFaFixedRefLimit
 
 
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
@@ -334,26 +341,64 @@ def test_global_attention(lib, wl):
     w_qkv, b_qkv, w_o, b_o = make_attention_weights(wl, 0)
     # second pass with 3x larger projection weights: the softmax becomes far from uniform
     # (random-init 0.02 weights alone give nearly flat attention, which would hide
-    # indexing mistakes)
+    # indexing mistakes) and the score bound of most rows passes the limit of the
+    # fixed-reference form, so the online form runs
     w_big = (w_qkv.float() * 3.0).to(torch.bfloat16)
     ctx = _ctx(lib, wl)
-    for wq in (w_qkv, w_big):
+    for tag, wq in (("stock", w_qkv), ("3x", w_big)):
         y = ctx.global_attn(xm.cuda(), wq.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
         ctx.poll()
         # each stage against the oracle fed with the GPU's own upstream (bf16) result
         ref_qkv = O.linear(to_f64(xm), to_f64(wq), to_f64(b_qkv))
         qkv = to_f64(ctx.debug_buffer(0))
-        assert rel_err(qkv, ref_qkv) <= bf16_bound(ref_qkv), "qkv projection"
+        check_bf16(f"{wl.name}/{tag}: qkv projection", qkv, ref_qkv)
+        b = score_bounds(qkv)
+        report(f"{wl.name}/{tag}: score bound", max=b.max(), share_fixed_reference=float((b <= FIXED_REF_LIMIT).mean()))
+        if tag == "stock":
+            assert b.max() <= FIXED_REF_LIMIT  # every row takes the fixed-reference form
+        else:
+            assert (b > FIXED_REF_LIMIT).mean() > 0.5  # most warps take the online form
         ref_o = O.attention_core(qkv, heads=16)
         o = to_f64(ctx.debug_buffer(1))
-        assert rel_err(o, ref_o) <= attention_core_bound(qkv, ref_o), "attention core"
+        check_bf16(f"{wl.name}/{tag}: attention core", o, ref_o, elem_noise=CORE_NOISE)
         ref_y = O.linear(o, to_f64(w_o), to_f64(b_o))
-        assert rel_err(to_f64(y), ref_y) <= bf16_bound(ref_y), "output projection"
-        if wq is w_qkv:  # end to end (bf16 intermediates on the GPU side, none in the oracle)
+        check_bf16(f"{wl.name}/{tag}: output projection", to_f64(y), ref_y)
+        if tag == "stock":  # end to end (bf16 intermediates on the GPU side, none in the oracle)
             ref_full = O.global_attention(to_f64(xm), to_f64(wq), to_f64(b_qkv), to_f64(w_o), to_f64(b_o), heads=16)
-            # three stored bf16 intermediates (qkv, o, y) instead of one rounding: the floor of
-            # the chain is about twice that of a single rounding at the 4-5 sigma entries
-            assert rel_err(to_f64(y), ref_full) <= 2 * bf16_bound(ref_full), "attention layer end to end"
+            check_bf16(f"{wl.name}: attention layer end to end", to_f64(y), ref_full, noise=LAYER_NOISE)
+    ctx.close()
+
+
+@pytest.mark.parametrize("grid,sharpness,form", [((22, 33), 4.0, "fixed"), ((22, 33), 8.0, "online"),
+                                                 ((34, 44), 4.0, "fixed")])
+def test_attention_core_with_peaked_softmax(lib, grid, sharpness, form):
+    """Rows in groups of near-duplicates spread through the sequence and query weights a multiple of
+    the key weights: a row's probability mass sits on itself and its group, so every key tile
+    matters.  sharpness 4 keeps the score bounds under the fixed-reference limit, 8 puts them over."""
+    ctx = lib.LiteVGGT(2, grid[0], grid[1], 0.0)  # merge ratio 0: M = N (1462 / 3002 rows, ragged tiles)
+    m = ctx.n_merged
+    assert m == ctx.n_tokens
+    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, 31 + m, groups=97, sharpness=sharpness)
+    y = ctx.global_attn(x.cuda(), w_qkv.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
+    ctx.poll()
+    qkv = to_f64(ctx.debug_buffer(0))
+    b = score_bounds(qkv)
+    report(f"peaked m={m} s={sharpness}: score bound", max=b.max(), min=b.min())
+    share_fixed = float((b <= FIXED_REF_LIMIT).mean())
+    assert share_fixed > 0.9 if form == "fixed" else share_fixed < 0.5
+    ref_o = O.attention_core(qkv, heads=16)
+    o = to_f64(ctx.debug_buffer(1))
+    check_bf16(f"peaked m={m} s={sharpness}: attention core", o, ref_o, elem_noise=CORE_NOISE)
+    # the case is what it claims to be: the rows of a query's own group hold most of its mass, so
+    # leaving out the keys of one tile (planted on the oracle's side) moves the result far beyond
+    # the tolerance
+    keep = np.ones(m, bool)
+    keep[256:384] = False
+    rows = np.flatnonzero(keep)[:200]
+    short = qkv[keep]
+    ref_short = O.attention_core(short, heads=16, rows=np.arange(200))
+    assert rel_err(o[rows], ref_short) > 20 * bf16_bound(ref_o)
+    check_bf16(f"peaked m={m} s={sharpness}: output projection", to_f64(y), O.linear(o, to_f64(w_o), to_f64(b_o)))
     ctx.close()
 
 
@@ -392,13 +437,18 @@ def test_global_attention_with_qk_norm_and_rope(lib, wl, mode):
     qkv = to_f64(ctx.debug_buffer(0))
     d = 1024
     for name, sl in (("Q", slice(0, d)), ("K", slice(d, 2 * d)), ("V", slice(2 * d, 3 * d))):
-        assert rel_err(qkv[:, sl], ref_qkv[:, sl]) <= 2 * bf16_bound(ref_qkv[:, sl]), f"{name} after {mode}"
+        # V is one rounding from the oracle's; Q and K were rounded once by the projection and once more
+        # after the transform: a second error of the size of the first, up to a quarter more in units of
+        # RMS after rotating pairs in which a small entry inherits the rounding of a large partner
+        second = 0.0 if name == "V" else 1.25 * rel_err(bf16_round(ref_qkv[:, sl]), ref_qkv[:, sl])
+        check_bf16(f"{wl.name}/{mode}: {name}", qkv[:, sl], ref_qkv[:, sl], noise=second)
     plain = to_f64(ctx.linear(xm, w_qkv.cuda(), b_qkv.cuda()))
     assert np.array_equal(qkv[:, 2 * d:], plain[:, 2 * d:])
     # the core on the GPU's own transformed Q/K/V, and the layer end to end
     ref_o = O.attention_core(qkv, heads=16)
-    assert rel_err(to_f64(ctx.debug_buffer(1)), ref_o) <= attention_core_bound(qkv, ref_o), "attention core"
-    assert rel_err(to_f64(y), ref_y) <= 3 * bf16_bound(ref_y), "layer end to end"
+    check_bf16(f"{wl.name}/{mode}: attention core", to_f64(ctx.debug_buffer(1)), ref_o, elem_noise=CORE_NOISE)
+    # one more stored rounding than the plain layer (the transformed Q and K)
+    check_bf16(f"{wl.name}/{mode}: layer end to end", to_f64(y), ref_y, noise=LAYER_NOISE)
     # and the options did something: Q is far from the plain projection
     assert rel_err(qkv[:, :d], plain[:, :d]) > 0.5
     plan.destroy()
@@ -418,15 +468,14 @@ def test_layernorm_frame_attention_and_mlp(lib, wl):
     xn = ctx.layernorm(x, g.cuda(), b.cuda(), eps=1e-6)
     ctx.poll()
     ref_n = O.layernorm(x64, to_f64(g), to_f64(b), 1e-6)
-    assert rel_err(to_f64(xn), ref_n) <= bf16_bound(ref_n)
+    check_bf16(f"{wl.name}: LayerNorm", to_f64(xn), ref_n)
     # frame-local attention on the GPU's own normalised rows, residual = the block input
     aw = [t.cuda() for t in w["attn"]]
     y = ctx.frame_attn(xn, *aw, residual=x)
     ctx.poll()
     ref_y = O.frame_attention(to_f64(xn), wl.frames, *[to_f64(t) for t in w["attn"]], heads=16, residual=x64)
-    # qkv, o and y are stored in bf16 on the way: twice the single-rounding bound, as for the
-    # global layer end to end
-    assert rel_err(to_f64(y), ref_y) <= 2 * bf16_bound(ref_y)
+    # qkv, o and y are stored in bf16 on the way, as for the global layer end to end
+    check_bf16(f"{wl.name}: frame attention layer", to_f64(y), ref_y, noise=LAYER_NOISE)
     # no token may see another frame: perturbing one frame must leave the others' rows bit-identical
     x2 = xn.clone()
     t = wl.tokens_per_frame
@@ -441,7 +490,7 @@ def test_layernorm_frame_attention_and_mlp(lib, wl):
     z = ctx.mlp(xn, *mw, residual=x)
     ctx.poll()
     ref_z = O.mlp(to_f64(xn), *[to_f64(t_) for t_ in w["mlp"]], residual=x64)
-    assert rel_err(to_f64(z), ref_z) <= 2 * bf16_bound(ref_z)
+    check_bf16(f"{wl.name}: MLP", to_f64(z), ref_z, noise=LAYER_NOISE)
     ctx.close()
 
 
@@ -463,7 +512,11 @@ def test_whole_layer_c1_and_host_entry(lib):
     ref_m = O.merge(x64, ex["dst_of"], ctx.n_merged)
     ref_y = O.global_attention(ref_m, *[to_f64(t) for t in w], heads=16)
     ref_out = O.unmerge(ref_y, ex["dst_of"], x64)
-    assert rel_err(to_f64(out), ref_out) <= bf16_bound(ref_out)
+    # the oracle is fed the GPU's plan but none of its intermediates; the residual dominates the
+    # output's scale, so the layer's stored intermediates stay inside the single-rounding bound
+    # (stated bound as it is; entry by entry the attention branch's stored intermediates show: its
+    # RMS is about half the output's, so half of LAYER_NOISE)
+    check_bf16("C1: whole layer (merge, attention, unmerge + residual)", to_f64(out), ref_out, elem_noise=LAYER_NOISE / 2)
     x_host = tok.clone().pin_memory()
     out_host = torch.empty_like(x_host).pin_memory()
     ctx.global_layer_host(plan, x_host, *w, out_host)
