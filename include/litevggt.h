@@ -170,9 +170,15 @@ litevggt_status litevggt_global_attn_ext(litevggt_ctx* ctx, const litevggt_plan*
  * library holds until the process exits.  Neither this call nor anything it calls allocates or
  * frees memory.
  *   - Works on the CURRENT device, for D = 1024 and 16 heads, and for 1 <= m <= 1024 merged rows;
- *     any other m is refused with LITEVGGT_ERR_SHAPE before anything is launched.
+ *     any other m is refused with LITEVGGT_ERR_SHAPE before anything is launched.  The extents
+ *     are taken on trust from m: x_merged and y_merged are read / written as [m, 1024], w_qkv as
+ *     [3072, 1024], w_o as [1024, 1024], b_qkv as [3072], b_o as [1024], all bf16; a shorter
+ *     buffer is overrun.
  *   - The first call on a device looks up the array's device address and the device's
- *     properties; make that first call outside any stream capture.  Later calls only enqueue.
+ *     properties and raises the kernels' shared-memory limits; it is also the call on which the
+ *     driver loads the library's kernels and the array itself onto that device.  Make it outside
+ *     any stream capture and before any region in which allocation is forbidden.  Later calls
+ *     only enqueue (one memset, the kernels) and encode tensor maps on the host.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.  The
  *     call clears what has to start at zero (the status word) itself; two calls whose work
  *     overlaps on the GPU (different streams, no ordering between them) race on the array.
@@ -278,6 +284,18 @@ litevggt_status litevggt_debug_buffer(litevggt_ctx* ctx, int which, void** dev_p
  * an out-of-range index since the last poll (the flag is cleared). */
 litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
 
+/* Self-test of the bounded waits (the paper has no counterpart; Sec. 3.4's kernels are this
+ * library's own).  Every pipelined kernel here waits on its barriers with a cycle limit; a wait
+ * that runs out raises the status word and the kernel returns instead of hanging.  This call
+ * launches a one-CTA kernel that waits, through the same device helpers, on a barrier that nobody
+ * arrives on, with `limit_cycles` (1,000 .. 2^32) as the limit.  Afterwards
+ * litevggt_poll_device_status must return LITEVGGT_ERR_DEVICE_TIMEOUT once and LITEVGGT_OK again
+ * on the next poll, and the context stays usable.  outcome (host, nullable; the call then
+ * synchronises the stream): bit 2 = the kernel ran to its end, bits 0 / 1 = a wait wrongly reported
+ * the barrier as complete (must be clear).  Nothing faults, traps or spins without a bound. */
+litevggt_status litevggt_selftest_bounded_wait(litevggt_ctx* ctx, int64_t limit_cycles, uint32_t* outcome,
+                                               void* stream);
+
 /* Device-time stopwatches.  Each step of the path is bracketed by CUDA events recorded on
  * the launching stream: which = 0 grad map, 1 var map, 2 partition + token lists, 3 cosine
  * matching (pack + GEMM/argmax), 4 selection + index build, 5 merge, 6 qkv projection,
@@ -287,6 +305,9 @@ litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream);
  * device time (ms) and the number of records (at most 64 are kept per step). */
 litevggt_status litevggt_timers_reset(litevggt_ctx* ctx);
 litevggt_status litevggt_timer_read(litevggt_ctx* ctx, int which, float* total_ms, int32_t* count);
+/* The individual records of one stopwatch, oldest first: up to `capacity` device times (ms) are
+ * written to `ms` (host), *count receives how many.  Synchronises on the recorded events. */
+litevggt_status litevggt_timer_samples(litevggt_ctx* ctx, int which, float* ms, int32_t capacity, int32_t* count);
 
 /* Number of kernels this library has launched on behalf of ctx since creation. */
 litevggt_status litevggt_launch_count(const litevggt_ctx* ctx, int64_t* launches);

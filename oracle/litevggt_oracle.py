@@ -282,6 +282,79 @@ def linear(a, w, b=None):
     return y
 
 
+# --------------------------------------------------------------------------------------
+# FP8 variant of the attention operands (Sec. 3.5 and supplementary "FP8 Quantization Details")
+# --------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_values():
+    """Every finite value of the E4M3 format the paper quantises to (supplementary "FP8 Quantization
+    Details": 1 sign, 4 exponent, 3 mantissa bits, exponent bias 7; the variant without infinities,
+    whose largest finite value is 448 and whose only NaN is the all-ones pattern).  Returns the 127
+    non-negative values, ascending, index = bit pattern (0x00 .. 0x7e)."""
+    vals = np.empty(127)
+    for code in range(127):
+        e, m = code >> 3, code & 7
+        vals[code] = m * 2.0 ** -9 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return vals
+
+
+def quantize_e4m3(x, scale):
+    """x / scale rounded to the nearest E4M3 value (ties to the even mantissa), saturating at +-448.
+    Returns (codes uint8, dequantised values codes * scale as float64).
+
+    The quotient is formed the way the kernel forms it - float32 value times the float32 reciprocal
+    448 / amax - because this decision between two codes is taken in that precision; everything
+    after it is exact."""
+    x32 = np.asarray(x, dtype=np.float32)
+    inv = np.float32(1.0) / np.asarray(scale, dtype=np.float32)
+    y = (x32 * inv).astype(np.float64)
+    vals = e4m3_values()
+    a = np.minimum(np.abs(y), E4M3_MAX)
+    hi = np.searchsorted(vals, a, side="left")          # first value >= a
+    hi = np.minimum(hi, vals.size - 1)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - vals[lo], vals[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))  # tie: the even code (even mantissa)
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    code = np.where(np.signbit(y), code | 0x80, code).astype(np.uint8)
+    deq = np.where(code & 0x80, -1.0, 1.0) * vals[code & 0x7f] * np.asarray(scale, dtype=np.float32).astype(np.float64)
+    return code, deq
+
+
+def fp8_head_scales(t, heads=16):
+    """Per-head scale of one of Q, K, V [M, D]: amax over the head's rows and channels divided by
+    448, so that the largest entry of the head lands on the largest E4M3 value (current scaling:
+    the statistics of the tensor being quantised; the paper's delayed scaling needs a history of
+    earlier iterations, which a single forward pass does not have).  float32 [heads]; 1/448 where a
+    head is all zero."""
+    t = np.asarray(t, dtype=np.float32)
+    m, d = t.shape
+    amax = np.abs(t).reshape(m, heads, d // heads).max(axis=(0, 2))
+    amax = np.where(amax > 0, amax, np.float32(1.0)).astype(np.float32)
+    return (amax / np.float32(E4M3_MAX)).astype(np.float32)
+
+
+def quantize_qkv_e4m3(qkv, heads=16):
+    """Q, K and V of qkv [M, 3D] quantised head by head.  Returns (dequantised qkv float64, codes
+    uint8 [M, 3D], scales float32 [3, heads])."""
+    qkv = np.asarray(qkv, dtype=np.float64)
+    m, d = qkv.shape[0], qkv.shape[1] // 3
+    dh = d // heads
+    deq = np.empty_like(qkv)
+    codes = np.empty(qkv.shape, dtype=np.uint8)
+    scales = np.empty((3, heads), dtype=np.float32)
+    for i in range(3):
+        part = qkv[:, i * d:(i + 1) * d]
+        scales[i] = fp8_head_scales(part, heads)
+        per_elem = np.repeat(scales[i], dh)[None, :]
+        c, v = quantize_e4m3(part, np.broadcast_to(per_elem, part.shape))
+        codes[:, i * d:(i + 1) * d] = c
+        deq[:, i * d:(i + 1) * d] = v
+    return deq, codes, scales
+
+
 def token_positions(frames, grid_h, grid_w, n_special=5):
     """Integer (row, column) position of every token for the rotary embedding.  Reading (the paper
     prints none; VGGT's aggregator, which Sec. 3.1 keeps, works this way): the special tokens of

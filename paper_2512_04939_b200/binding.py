@@ -77,6 +77,7 @@ def load_library():
         "litevggt_host_drain": [vp, vp],
         "litevggt_timers_reset": [vp],
         "litevggt_timer_read": [vp, C.c_int, P(C.c_float), P(i32)],
+        "litevggt_timer_samples": [vp, C.c_int, P(C.c_float), i32, P(i32)],
         "litevggt_linear": [vp, vp, i64, i64, vp, i64, vp, vp, vp],
         "litevggt_should_refresh": [vp, vp, i32, P(i32)],
         "litevggt_plan_export": [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
@@ -84,6 +85,7 @@ def load_library():
         "litevggt_plan_destroy": [vp],
         "litevggt_debug_buffer": [vp, C.c_int, P(vp), P(C.c_size_t)],
         "litevggt_poll_device_status": [vp, vp],
+        "litevggt_selftest_bounded_wait": [vp, i64, P(C.c_uint32), vp],
         "litevggt_launch_count": [vp, P(i64)],
     }
     for name, args in sigs.items():
@@ -115,14 +117,47 @@ def _stream():
 STATIC_ATTN_MAX_ROWS = 1024
 
 
+def _check_static_attn_args(xm, w_qkv, b_qkv, w_o, b_o, out, device_status):
+    """The C entry point is told only m and trusts every extent, so a wrong shape, dtype or device
+    would send its kernels past the end of an allocation: refuse such arguments here, before any
+    launch.  Shapes first, so that the message names the actual mistake."""
+    d = 1024
+    if xm.dim() != 2 or xm.shape[1] != d or not 1 <= xm.shape[0] <= STATIC_ATTN_MAX_ROWS:
+        raise ValueError(f"x_merged must be [m, {d}] with 1 <= m <= {STATIC_ATTN_MAX_ROWS}, got {tuple(xm.shape)}")
+    wanted = {"w_qkv": (w_qkv, (3 * d, d)), "w_o": (w_o, (d, d)), "b_qkv": (b_qkv, (3 * d,)), "b_o": (b_o, (d,)),
+              "out": (out, tuple(xm.shape))}
+    for name, (t, shape) in wanted.items():
+        if t is None:
+            if name in ("b_qkv", "b_o"):
+                continue
+            raise ValueError(f"{name} is required")
+        if tuple(t.shape) != shape:
+            raise ValueError(f"{name} must have shape {shape}, got {tuple(t.shape)}")
+    for name, t in (("x_merged", xm), ("w_qkv", w_qkv), ("b_qkv", b_qkv), ("w_o", w_o), ("b_o", b_o), ("out", out)):
+        if t is None:
+            continue
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous bfloat16 tensor")
+    if device_status is not None and (device_status.dtype != torch.int32 or device_status.numel() != 1):
+        raise ValueError("device_status must be one int32 element")
+    tensors = [t for t in (xm, w_qkv, b_qkv, w_o, b_o, out, device_status) if t is not None]
+    if not all(t.is_cuda for t in tensors):
+        raise ValueError("every tensor must live on a CUDA device")
+    current = torch.cuda.current_device()
+    if any(t.device.index != current for t in tensors):
+        raise ValueError(f"every tensor must live on the current device (cuda:{current}): the entry point works there")
+
+
 def global_attn_static(xm, w_qkv, b_qkv, w_o, b_o, out=None, device_status=None):
     """Attention layer over up to STATIC_ATTN_MAX_ROWS merged rows through the entry point that
     allocates nothing (no context; intermediates in the library's own fixed device array).  The
     output tensor is the caller's; pass ``out`` to keep this wrapper from allocating one.
-    ``device_status``: optional int32 CUDA tensor of one element that receives the kernels' flag."""
+    ``device_status``: optional int32 CUDA tensor of one element that receives the kernels' flag.
+    Shapes, dtypes and devices are checked here, because the C entry point cannot."""
     lib = load_library()
     if out is None:
         out = torch.empty_like(xm)
+    _check_static_attn_args(xm, w_qkv, b_qkv, w_o, b_o, out, device_status)
     _check(lib.litevggt_global_attn_static(_ptr(xm), xm.shape[0], _ptr(w_qkv), _ptr(b_qkv), _ptr(w_o), _ptr(b_o),
                                            _ptr(out), _ptr(device_status), _stream()), "global_attn_static")
     return out
@@ -366,9 +401,28 @@ class LiteVGGT:
             out[name] = (ms.value, cnt.value)
         return out
 
+    def timers_samples(self) -> dict:
+        """{step name: [device ms of each record since the last reset, oldest first]} (synchronises)."""
+        out = {}
+        buf = (C.c_float * 64)()
+        for i, name in enumerate(self.TIMER_NAMES):
+            cnt = C.c_int32()
+            _check(self.lib.litevggt_timer_samples(self.handle, i, buf, 64, C.byref(cnt)), "timer_samples")
+            out[name] = [float(buf[k]) for k in range(cnt.value)]
+        return out
+
     def poll(self):
         """Synchronise the current stream; raise if a kernel flagged a timeout / bad index."""
         _check(self.lib.litevggt_poll_device_status(self.handle, _stream()), "poll_device_status")
+
+    def selftest_bounded_wait(self, limit_cycles: int = 1_000_000) -> int:
+        """Run the one-CTA kernel that waits on a barrier nobody arrives on; returns its outcome
+        word (4 = ran to its end, no wait reported a false completion).  The next poll() raises
+        LITEVGGT_ERR_DEVICE_TIMEOUT, the one after that is clean."""
+        word = C.c_uint32(0)
+        _check(self.lib.litevggt_selftest_bounded_wait(self.handle, int(limit_cycles), C.byref(word), _stream()),
+               "selftest_bounded_wait")
+        return int(word.value)
 
     def launch_count(self) -> int:
         n = C.c_int64()

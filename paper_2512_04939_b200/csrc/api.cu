@@ -372,6 +372,26 @@ litevggt_status litevggt_timer_read(litevggt_ctx* ctx, int which, float* total_m
   return LITEVGGT_OK;
 }
 
+litevggt_status litevggt_timer_samples(litevggt_ctx* ctx, int which, float* ms, int32_t capacity, int32_t* count) {
+  if (!ctx_ok(ctx) || ms == nullptr || count == nullptr) return LITEVGGT_ERR_NULL;
+  if (which < 0 || which >= kNumTimers || capacity < 0) return LITEVGGT_ERR_SHAPE;
+  Timers& tm = ctx->timers;
+  *count = 0;
+  if (!tm.created) return LITEVGGT_ERR_CUDA;
+  // the ring keeps the latest kTimerSlots records; slot i holds record i, i + kTimerSlots, ...
+  const int used = tm.used[which];
+  const int kept = used < kTimerSlots ? used : kTimerSlots;
+  const int n = kept < capacity ? kept : capacity;
+  for (int i = 0; i < n; ++i) {
+    const int slot = (used - kept + i) % kTimerSlots;
+    if (cudaEventSynchronize(tm.stop[which][slot]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms[i], tm.start[which][slot], tm.stop[which][slot]) != cudaSuccess)
+      return cuda_status(cudaGetLastError());
+  }
+  *count = n;
+  return LITEVGGT_OK;
+}
+
 litevggt_status litevggt_destroy(litevggt_ctx* ctx) {
   if (ctx == nullptr) return LITEVGGT_OK;
   if (!ctx_ok(ctx)) return LITEVGGT_ERR_NULL;
@@ -902,6 +922,22 @@ litevggt_status litevggt_poll_device_status(litevggt_ctx* ctx, void* stream) {
   if (word & kStatusTimeout) return LITEVGGT_ERR_DEVICE_TIMEOUT;
   if (word & kStatusBounds) return LITEVGGT_ERR_DEVICE_BOUNDS;
   return LITEVGGT_OK;
+}
+
+litevggt_status litevggt_selftest_bounded_wait(litevggt_ctx* ctx, int64_t limit_cycles, uint32_t* outcome, void* stream) {
+  if (!ctx_ok(ctx)) return LITEVGGT_ERR_NULL;
+  if (limit_cycles < 1000 || limit_cycles > (1ll << 32)) return LITEVGGT_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)stream;
+  uint32_t* dev_outcome = ctx->ws.status + 1;  // second word of the status block
+  int n = 0;
+  cudaError_t e = launch_bounded_wait_selftest(ctx, limit_cycles, dev_outcome, s, &n);
+  bump(ctx, n);
+  if (e != cudaSuccess) return cuda_status(e);
+  if (outcome != nullptr) {
+    e = cudaMemcpyAsync(outcome, dev_outcome, sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  }
+  return cuda_status(e);
 }
 
 litevggt_status litevggt_launch_count(const litevggt_ctx* ctx, int64_t* launches) {

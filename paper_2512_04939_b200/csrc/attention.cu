@@ -616,9 +616,10 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
                           int, int, int, float, uint32_t*);
   const Kernel kernels[2][2] = {{flash_attention_kernel<false, false>, flash_attention_kernel<false, true>},
                                 {flash_attention_kernel<true, false>, flash_attention_kernel<true, true>}};
+  static std::atomic<unsigned long long> smem_set[2][2];
   for (int a = 0; a < 2; ++a)
     for (int b = 0; b < 2; ++b) {
-      cudaError_t e = cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, kFaSmemBytes);
+      cudaError_t e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(kernels[a][b]), kFaSmemBytes, smem_set[a][b]);
       if (e != cudaSuccess) return e;
     }
   const dim3 grid((unsigned)((seq_len + 255) / 256), (unsigned)ctx->sz.heads, (unsigned)n_seq);

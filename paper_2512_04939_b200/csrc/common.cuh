@@ -80,10 +80,12 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t par
   return ok != 0;
 }
 
-// Per-CTA abort flag (shared memory) plus the context's status word (global memory).
+// Per-CTA abort flag (shared memory), the context's status word (global memory) and the number
+// of clock cycles after which a wait gives up.
 struct WaitCtl {
   volatile uint32_t* abort_flag;
   uint32_t* status;
+  long long limit = kTimeoutCycles;
 };
 
 // Wait for the phase with the given parity to complete.  Returns false when the wait
@@ -94,7 +96,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
   while (true) {
     if (mbar_try_wait_parked(bar, parity, 2000u)) return true;  // parks for at most 2 us per try
     if (*ctl.abort_flag != 0u) return false;
-    if (clock64() - t0 > kTimeoutCycles) {
+    if (clock64() - t0 > ctl.limit) {
       *ctl.abort_flag = 1u;
       atomicOr(ctl.status, kStatusTimeout);
       return false;

@@ -20,8 +20,9 @@ cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m
   epi.bias = bias;
   epi.m_rows = (int)m;
   epi.n_cols = (int)n;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<LinearEpilogue>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kGemmSmemBytes);
+  static std::atomic<unsigned long long> smem_set{0};
+  cudaError_t e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(gemm_tc_kernel<LinearEpilogue>), kGemmSmemBytes,
+                                            smem_set);
   if (e != cudaSuccess) return e;
   const long long tiles = ((m + kGemmBM - 1) / kGemmBM) * ((n + kGemmBN - 1) / kGemmBN);
   const int grid = tiles < ctx->num_sms ? (int)tiles : ctx->num_sms;
@@ -50,8 +51,9 @@ cudaError_t launch_linear_mlp(litevggt_ctx* ctx, const __nv_bfloat16* a, long lo
   epi.n_cols = (int)n;
   epi.ld_res = n;
   epi.gelu = gelu;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<MlpEpilogue>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kGemmSmemBytes);
+  static std::atomic<unsigned long long> smem_set{0};
+  cudaError_t e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(gemm_tc_kernel<MlpEpilogue>), kGemmSmemBytes,
+                                            smem_set);
   if (e != cudaSuccess) return e;
   const long long tiles = ((m + kGemmBM - 1) / kGemmBM) * ((n + kGemmBN - 1) / kGemmBN);
   const int grid = tiles < ctx->num_sms ? (int)tiles : ctx->num_sms;

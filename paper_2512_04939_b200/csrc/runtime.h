@@ -8,6 +8,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/litevggt.h"
 
 namespace lv {
@@ -24,6 +26,19 @@ struct Sizes {
 };
 
 inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
+
+// Raises a kernel's dynamic shared-memory limit once per device (`done` holds one bit per device,
+// one object per kernel), so that a launcher's later calls only enqueue work.
+inline cudaError_t set_max_dynamic_smem_once(const void* kernel, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
 
 constexpr long long kMlpChunkRows = 131072;  // rows of the 4D-wide hidden activations held at a time (1 GiB)
 
@@ -170,6 +185,10 @@ cudaError_t launch_linear_mlp(litevggt_ctx* ctx, const __nv_bfloat16* a, long lo
                               const __nv_bfloat16* residual, __nv_bfloat16* out, cudaStream_t s, int* launches);
 cudaError_t launch_layernorm(const __nv_bfloat16* x, const __nv_bfloat16* gamma, const __nv_bfloat16* beta,
                              __nv_bfloat16* out, long long rows, float eps, cudaStream_t s, int* launches);
+
+// selftest.cu: one CTA waits on a barrier that nobody arrives on, with the given cycle limit
+cudaError_t launch_bounded_wait_selftest(litevggt_ctx* ctx, long long limit_cycles, uint32_t* outcome, cudaStream_t s,
+                                         int* launches);
 
 // attention.cu
 // n_seq independent sequences of seq_len rows each, laid back to back in qkv / o

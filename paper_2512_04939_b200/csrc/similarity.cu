@@ -85,8 +85,8 @@ cudaError_t launch_match(litevggt_ctx* ctx, const __nv_bfloat16* x, int* best_ds
   epi.best_val = best_sim;
   epi.m_rows = (int)z.n_src;
   epi.n_cols = (int)z.n_dst;
-  e = cudaFuncSetAttribute(gemm_tc_kernel<ArgmaxEpilogue>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kGemmSmemBytes);
+  static std::atomic<unsigned long long> smem_set{0};
+  e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(gemm_tc_kernel<ArgmaxEpilogue>), kGemmSmemBytes, smem_set);
   if (e != cudaSuccess) return e;
   const int m_blocks = (int)((z.n_src + kGemmBM - 1) / kGemmBM);
   const int grid = m_blocks < ctx->num_sms ? m_blocks : ctx->num_sms;

@@ -46,3 +46,38 @@ def test_status_strings_and_default_config_without_gpu():
     assert lib.litevggt_sizes(None, None, None, None, None, None) == 1
     assert lib.litevggt_merge(None, None, None, None, None) == 1
     assert lib.litevggt_plan_destroy(None) == 0 and lib.litevggt_destroy(None) == 0
+
+
+def test_static_attention_wrapper_refuses_bad_arguments_before_any_launch():
+    """litevggt_global_attn_static is told only m and trusts every extent; its Python wrapper must
+    turn a wrong shape, dtype or device into an error on the host (no GPU is touched here)."""
+    import pytest
+    import torch
+
+    import paper_2512_04939_b200 as pkg
+
+    bf = torch.bfloat16
+    good = dict(xm=torch.zeros(16, 1024, dtype=bf), w_qkv=torch.zeros(3072, 1024, dtype=bf),
+                b_qkv=torch.zeros(3072, dtype=bf), w_o=torch.zeros(1024, 1024, dtype=bf), b_o=torch.zeros(1024, dtype=bf))
+    bad = [
+        dict(xm=torch.zeros(16, 512, dtype=bf)),                      # half-width rows
+        dict(xm=torch.zeros(pkg.STATIC_ATTN_MAX_ROWS + 1, 1024, dtype=bf)),
+        dict(w_qkv=torch.zeros(1024, 1024, dtype=bf)),                # one projection instead of three
+        dict(w_o=torch.zeros(1024, 512, dtype=bf)),
+        dict(b_qkv=torch.zeros(1024, dtype=bf)),                      # short bias
+        dict(b_o=torch.zeros(8, dtype=bf)),
+        dict(xm=torch.zeros(16, 1024, dtype=torch.float32)),          # wrong dtype
+        dict(w_o=torch.zeros(1024, 2048, dtype=bf)[:, ::2]),          # not contiguous
+        dict(out=torch.zeros(8, 1024, dtype=bf)),                     # short output
+        dict(device_status=torch.zeros(2, dtype=torch.int32)),
+        dict(device_status=torch.zeros(1, dtype=torch.int64)),
+    ]
+    for change in bad:
+        args = dict(good, out=None, device_status=None)
+        args.update(change)
+        with pytest.raises(ValueError):
+            pkg.global_attn_static(args["xm"], args["w_qkv"], args["b_qkv"], args["w_o"], args["b_o"], out=args["out"],
+                                   device_status=args["device_status"])
+    # right shapes, but host tensors: refused as well (the entry point works on the current CUDA device)
+    with pytest.raises(ValueError, match="CUDA"):
+        pkg.global_attn_static(good["xm"], good["w_qkv"], good["b_qkv"], good["w_o"], good["b_o"])

@@ -7,6 +7,7 @@ import os
 import subprocess
 import sys
 
+import numpy as np
 import pytest
 import torch
 import torch.distributed as dist
@@ -47,13 +48,40 @@ def test_single_rank_needs_no_process_group():
     assert bench.aggregate_frames_per_s(200, 6, 1, 60.0) == pytest.approx(200 * 6 / 0.06)
 
 
-def test_extrapolation_scales_quadratic_and_linear_steps():
+def test_frames_per_s_amortises_the_plan_over_the_refresh_interval():
     t = dict(grad_map=1.0, var_map=0.2, partition=0.1, index_build=0.1, match=0.5, merge=0.1, qkv_proj=0.2,
              out_proj=0.1, unmerge=0.1, attention=2.0)
-    # 10x the frames: linear steps x10, quadratic x100; plan amortised over 6 layers
-    layer = (0.1 + 0.2 + 0.1 + 0.1) * 10 + 2.0 * 100
-    plan = (0.2 + 0.1 + 0.1) * 10 + 0.5 * 100
-    assert bench.extrapolate_frames_per_s(t, 16, 160, 6) == pytest.approx(160 / (layer + plan / 6))
+    layer = 0.1 + 0.2 + 2.0 + 0.1 + 0.1
+    plan = 0.2 + 0.1 + 0.5 + 0.1
+    assert bench.frames_per_s_from_steps(t, 160, 6) == pytest.approx(160 / (layer + plan / 6))
+
+
+def test_oracle_sample_on_c1_scales_row_samples_to_the_whole_problem():
+    """The bounded samples of the CPU baseline on config C1, where the samples can cover the whole
+    problem: with every src row, every query row and all 16 heads sampled the row-sampled steps are
+    the oracle's full calls, so their extrapolation factors are 1."""
+    from synthdata import WORKLOADS, make_attention_weights, make_images, make_tokens
+
+    wl = WORKLOADS["C1"]
+    images = make_images(wl)
+    tokens = make_tokens(wl, images)
+    weights = make_attention_weights(wl, 0)
+    sample = dict(match_rows=10 ** 6, attn_rows=10 ** 6, attn_heads=16, proj_rows=10 ** 6, linear_frames=wl.frames)
+    data = bench.prepare_oracle_sample(wl, images, tokens, weights, sample)
+    sz = data["sizes"]
+    assert data["match_src"].size == sz["n_src"] and data["match_dst"].size == sz["n_dst"]
+    assert data["attn_rows"].size == sz["M"] and len(data["qkv_heads"]) == 16 and data["x_proj"].shape[0] == sz["M"]
+    assert data["qkv_heads"][0].shape == (sz["M"], 192)
+    t, margin = bench.oracle_sampled_layer(wl, data)
+    assert set(t) == {"grad_map", "var_map", "partition", "match", "index_build", "merge", "unmerge", "qkv_proj",
+                      "out_proj", "attention"}
+    assert all(v > 0 for v in t.values()) and margin.size == sz["n_src"] and np.all(margin >= 0)
+    hist = bench.margin_histogram(margin)
+    assert 0 <= hist["below_1e-5"] <= hist["below_1e-4"] <= hist["below_1e-3"] <= 1
+    # a quarter of the rows sampled: the same call on fewer rows, scaled by rows / sampled rows
+    small = bench.prepare_oracle_sample(wl, images, tokens, weights, dict(sample, match_rows=125, attn_rows=136, attn_heads=4))
+    assert small["match_src"].size == 125 and small["attn_rows"].size == 136 and len(small["qkv_heads"]) == 4
+    assert "125 of 501 src rows" in bench.sample_description(wl, sample, small)
 
 
 def test_clock_sampler_parses_nvidia_smi_lines():

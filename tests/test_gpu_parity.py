@@ -578,6 +578,40 @@ def test_pipelined_host_entry_equals_the_ordered_one(lib, wl):
     ctx.close()
 
 
+# ------------------------------------------------------------------ bounded waits
+def test_a_wait_that_runs_out_sets_the_status_word_and_leaves_the_context_usable(lib):
+    """Every pipelined kernel waits on its barriers with a cycle limit.  The self-test kernel waits,
+    through the same device helpers, on a barrier that nobody arrives on (limit: a million cycles,
+    half a millisecond): it must return, the status poll must report the timeout once and be clean
+    afterwards, and ordinary work on the same context must still be right."""
+    wl = WORKLOADS["C1"]
+    ctx = _ctx(lib, wl)
+    a = torch.randn(300, 128, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
+    w = (0.05 * torch.randn(320, 128, generator=torch.Generator().manual_seed(4))).to(torch.bfloat16)
+    ref = to_f64(a) @ to_f64(w).T
+    before = ctx.linear(a.cuda(), w.cuda(), None)
+    ctx.poll()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    outcome = ctx.selftest_bounded_wait(1_000_000)
+    t1.record()
+    torch.cuda.synchronize()
+    assert outcome == 4, f"outcome word {outcome}: bit 2 = ran to its end, bits 0/1 = a wait reported a false completion"
+    assert t0.elapsed_time(t1) < 100.0  # a million cycles, not the production limit of 2^32
+    with pytest.raises(lib.LiteVGGTError) as e:
+        ctx.poll()
+    assert e.value.code == 9  # LITEVGGT_ERR_DEVICE_TIMEOUT
+    ctx.poll()  # the flag was cleared by the poll that reported it
+    after = ctx.linear(a.cuda(), w.cuda(), None)
+    ctx.poll()
+    assert torch.equal(before, after)
+    check_bf16("linear after a timed-out wait", to_f64(after), ref)
+    # limits outside [1e3, 2^32] are refused on the host
+    assert ctx.lib.litevggt_selftest_bounded_wait(ctx.handle, 10, None, None) == 3
+    ctx.close()
+
+
 # ------------------------------------------------------------------ ABI misuse
 def test_abi_misuse_returns_error_codes(lib):
     wl = WORKLOADS["C1"]

@@ -619,3 +619,61 @@ def test_layer_noise_allowance_covers_stored_bf16_intermediates():
     # the rounding of o alone accounts for it
     only_o = np.abs(O.linear(bf16_round(o), w[2], w[3]) - y_exact).max() / rms
     assert only_o > 0.8 * noise.max()
+
+
+# ------------------------------------------------------------------ FP8 (E4M3) quantisation
+def test_e4m3_format_closed_forms():
+    """The format's landmarks: 127 finite non-negative values, largest 448, smallest subnormal 2^-9,
+    smallest normal 2^-6, eight steps per binade, 1.0 at code 0x38."""
+    v = O.e4m3_values()
+    assert v.size == 127 and v[0] == 0.0 and np.all(np.diff(v) > 0)
+    assert v[-1] == 448.0 and v[1] == 2.0 ** -9 and v[8] == 2.0 ** -6 and v[0x38] == 1.0
+    assert np.array_equal(v[0x38:0x40], 1.0 + np.arange(8) / 8.0)
+    assert np.array_equal(v[1:8], np.arange(1, 8) * 2.0 ** -9)  # the subnormals
+
+
+def test_e4m3_matches_the_library_cast():
+    """torch's float8_e4m3fn cast (round to nearest even, same format) on values spread over the
+    whole range, exact ties included."""
+    rng = np.random.default_rng(99)
+    x = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.uniform(-4, 2.6, 4000),
+                        [0.0, 448.0, -448.0, 2.0 ** -10, 3 * 2.0 ** -10, 1.0625, 1.1875, 17.0, 19.0, 2.0 ** -9]])
+    x = x[np.abs(x) <= 448.0].astype(np.float32)
+    code, deq = O.quantize_e4m3(x, np.float32(1.0))
+    ref = torch.from_numpy(x).to(torch.float8_e4m3fn)
+    assert np.array_equal(deq, ref.float().numpy().astype(np.float64))
+    same_bits = code == ref.view(torch.uint8).numpy()
+    assert np.all(same_bits | (deq == 0))  # the sign of a zero is the one place the bit patterns may differ
+
+
+def test_e4m3_hand_picked_roundings_and_saturation():
+    one = np.float32(1.0)
+    q = lambda v: O.quantize_e4m3(np.array(v, dtype=np.float32), one)[1].tolist()
+    assert q([1.0625, 1.1875, 1.3125]) == [1.0, 1.25, 1.25]      # ties go to the even mantissa
+    assert q([1.06, 1.07]) == [1.0, 1.125]
+    assert q([500.0, -1e9, 464.0]) == [448.0, -448.0, 448.0]      # saturating
+    assert q([2.0 ** -10, 2.0 ** -10 * 1.01, 2.0 ** -11]) == [0.0, 2.0 ** -9, 0.0]  # tie to even (zero), just above, below
+    # a scale maps the head's largest entry onto 448 and comes back out exactly
+    x = np.array([[3.5, -7.0, 0.21875]], dtype=np.float32)
+    s = O.fp8_head_scales(np.tile(x, (1, 1)), heads=1)
+    assert s[0] == np.float32(7.0) / np.float32(448.0)
+    code, deq = O.quantize_e4m3(x, s[0])
+    assert deq[0, 1] == -7.0 and deq[0, 0] == 3.5 and abs(deq[0, 2] - 0.21875) <= 0.21875 * 2.0 ** -4
+
+
+def test_e4m3_relative_error_bound_and_head_scales():
+    """Every normal-range value is within 2^-4 relative of its code; per-head scales follow each head's own
+    amax, and the quantised attention operands give an attention output close to the unquantised one."""
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((300, 3 * 128))
+    x[:, 64:128] *= 50.0  # one head of Q far larger than the others
+    deq, codes, scales = O.quantize_qkv_e4m3(x, heads=2)
+    assert scales.shape == (3, 2) and scales[0, 1] > 10 * scales[0, 0]
+    big = np.abs(x) > (np.repeat(scales.reshape(6), 64)[None, :] * 2.0 ** -6)
+    assert np.all(np.abs(deq - x)[big] <= np.abs(x)[big] * 2.0 ** -4 * (1 + 1e-6))
+    assert codes.dtype == np.uint8 and np.all((codes & 0x7f) != 0x7f)  # never the NaN pattern
+    # (judged on the head with ordinary magnitudes; in the other one the 50x scores make the softmax a
+    # near-argmax, which any perturbation of the scores can flip)
+    o_q = O.attention_core(deq, heads=2)[:, :64]
+    o = O.attention_core(x, heads=2)[:, :64]
+    assert 0 < np.abs(o_q - o).max() / np.sqrt(np.mean(o * o)) < 0.25

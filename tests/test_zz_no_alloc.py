@@ -10,8 +10,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as O
 from synthdata import WORKLOADS, make_attention_weights
-from helpers import bf16_bound, rel_err, to_f64
+from helpers import LAYER_NOISE, bf16_bound, check_bf16, rel_err, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -38,13 +39,28 @@ def test_static_attention_matches_context_attention_twice():
         # fact identical bits
         assert rel_err(to_f64(got), ref) <= bf16_bound(ref), f"call {call}"
         assert torch.equal(got, want), f"call {call}"
-    # a shorter sequence right after a longer one: rows left in the array must not leak in
-    xs = xm[:200].contiguous()
+    # a shorter sequence right after a longer one: rows left in the array must not leak in, so the
+    # result is judged against the CPU oracle on the 200 rows alone
+    # (unit-variance rows: with the 2.5x rows above the scores are large enough for the bf16 rounding of
+    # q and k alone to move the probabilities by several per cent, which no end-to-end bound covers)
+    xs = torch.randn(200, 1024, generator=gen).to(torch.bfloat16).cuda()
     got = pkg.global_attn_static(xs, w_qkv, None, w_o, None)
-    again = pkg.global_attn_static(xs, w_qkv, None, w_o, None)
     torch.cuda.synchronize()
-    assert torch.equal(got, again)
-    assert torch.isfinite(got.float()).all()
+    ref_y = O.global_attention(to_f64(xs), to_f64(w_qkv), None, to_f64(w_o), None, heads=16)
+    check_bf16("static entry point, 200 rows after 543", to_f64(got), ref_y, noise=LAYER_NOISE)
+    # and the call allocates nothing: with the output given, neither the driver's free memory nor
+    # the caching allocator's books move across a call
+    out = torch.empty_like(xs)
+    pkg.global_attn_static(xs, w_qkv, None, w_o, None, out=out)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    booked_before = torch.cuda.memory_allocated()
+    reserved_before = torch.cuda.memory_reserved()
+    pkg.global_attn_static(xs, w_qkv, None, w_o, None, out=out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert torch.cuda.memory_allocated() == booked_before and torch.cuda.memory_reserved() == reserved_before
+    assert torch.equal(out, got)
     ctx.close()
 
 
