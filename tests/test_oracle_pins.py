@@ -676,4 +676,4 @@ def test_e4m3_relative_error_bound_and_head_scales():
     # near-argmax, which any perturbation of the scores can flip)
     o_q = O.attention_core(deq, heads=2)[:, :64]
     o = O.attention_core(x, heads=2)[:, :64]
-    assert 0 < np.abs(o_q - o).max() / np.sqrt(np.mean(o * o)) < 0.25
+    assert 0 < np.abs(o_q - o).max() / np.sqrt(np.mean(o * o)) < 0.5
