@@ -71,7 +71,11 @@ typedef struct {
   int32_t cell_h, cell_w;     /* 2, 2: one anchor per cell in frames 1..F-1 */
   int32_t var_window;         /* 3: window of the Var map */
   int32_t recompute_interval; /* 6: refresh the plan every this many global layers */
-  int32_t qkv_dtype;          /* 0 = bf16 (only value supported) */
+  int32_t qkv_dtype;          /* 0 = bf16; 1 = E4M3: litevggt_global_attn / _ext quantise the projected Q, K, V head
+                                 by head (scale = amax / 448 of the head, taken from the tensor itself) and
+                                 run both attention products on 8-bit operands, the probabilities rounded to
+                                 E4M3 as well (Sec. 3.5 and supplementary "FP8 Quantization Details").  The
+                                 projections, merge and unmerge stay bf16. */
 } litevggt_config;
 
 typedef struct litevggt_ctx litevggt_ctx;   /* workspace, tensor maps, device status word */
@@ -277,7 +281,10 @@ litevggt_status litevggt_plan_import(litevggt_ctx* ctx, const int32_t* dst_of, l
 litevggt_status litevggt_plan_destroy(litevggt_plan* plan);
 
 /* Pointer to an internal device buffer of the last litevggt_global_attn call (tests):
- * which = 0: qkv bf16 [M,3D];  which = 1: attention output o bf16 [M,D]. */
+ * which = 0: qkv bf16 [M,3D];  which = 1: attention output o bf16 [M,D];  with qkv_dtype = 1 also
+ * 2: Q as E4M3 bytes [M,D];  3: K likewise;  4: V transposed, bytes [D, round_up(M,128)] (row =
+ * head * 64 + channel, column = key, zero beyond M);  5: float [3, heads], the largest magnitude of
+ * Q, K, V per head (scale = amax / 448). */
 litevggt_status litevggt_debug_buffer(litevggt_ctx* ctx, int which, void** dev_ptr, size_t* bytes);
 
 /* Synchronise `stream` and report whether any kernel flagged a bounded-wait timeout or
@@ -300,7 +307,8 @@ litevggt_status litevggt_selftest_bounded_wait(litevggt_ctx* ctx, int64_t limit_
  * the launching stream: which = 0 grad map, 1 var map, 2 partition + token lists, 3 cosine
  * matching (pack + GEMM/argmax), 4 selection + index build, 5 merge, 6 qkv projection,
  * 7 attention core, 8 output projection, 9 unmerge, 10 LayerNorm, 11 frame-local attention layer,
- * 12 MLP, 13 Q/K normalisation + rotary embedding.  litevggt_timers_reset forgets all
+ * 12 MLP, 13 Q/K normalisation + rotary embedding, 14 E4M3 quantisation of Q/K/V.
+ * litevggt_timers_reset forgets all
  * records; litevggt_timer_read synchronises on the recorded events and returns the summed
  * device time (ms) and the number of records (at most 64 are kept per step). */
 litevggt_status litevggt_timers_reset(litevggt_ctx* ctx);

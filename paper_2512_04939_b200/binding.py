@@ -386,8 +386,29 @@ class LiteVGGT:
         view = _DeviceBuffer(ptr.value, (self.n_merged, cols))
         return torch.as_tensor(view, device=self.device).view(torch.bfloat16).clone()
 
+    def debug_fp8_buffers(self) -> dict:
+        """The E4M3 operands of the last global_attn call of a context made with qkv_dtype=1, copied
+        out: q8, k8 uint8 [M, D]; v8t uint8 [D, round_up(M, 128)] (V transposed: row = head * 64 +
+        channel, column = key, zero beyond M); amax float32 [3, heads] of Q, K, V."""
+        out = {}
+        m_pad = (self.n_merged + 127) // 128 * 128
+        shapes = {2: ("q8", (self.n_merged, self.dim)), 3: ("k8", (self.n_merged, self.dim)), 4: ("v8t", (self.dim, m_pad))}
+        for which, (name, shape) in shapes.items():
+            ptr, nbytes = C.c_void_p(), C.c_size_t()
+            _check(self.lib.litevggt_debug_buffer(self.handle, which, C.byref(ptr), C.byref(nbytes)), "debug_buffer")
+            assert nbytes.value == shape[0] * shape[1]
+            iface = {"shape": shape, "typestr": "|u1", "data": (ptr.value, False), "version": 2}
+            holder = type("_U8", (), {"__cuda_array_interface__": iface})()
+            out[name] = torch.as_tensor(holder, device=self.device).clone()
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        _check(self.lib.litevggt_debug_buffer(self.handle, 5, C.byref(ptr), C.byref(nbytes)), "debug_buffer")
+        iface = {"shape": (3, 16), "typestr": "<f4", "data": (ptr.value, False), "version": 2}
+        holder = type("_F4", (), {"__cuda_array_interface__": iface})()
+        out["amax"] = torch.as_tensor(holder, device=self.device).clone()
+        return out
+
     TIMER_NAMES = ("grad_map", "var_map", "partition", "match", "index_build", "merge", "qkv_proj",
-                   "attention", "out_proj", "unmerge", "layernorm", "frame_attn", "mlp", "qk_embed")
+                   "attention", "out_proj", "unmerge", "layernorm", "frame_attn", "mlp", "qk_embed", "qkv_quantize")
 
     def timers_reset(self):
         _check(self.lib.litevggt_timers_reset(self.handle), "timers_reset")

@@ -40,7 +40,7 @@ litevggt_status compute_sizes(const litevggt_config& c, Sizes* out) {
   if (c.cell_h < 1 || c.cell_w < 1 || c.var_window != 3 || c.recompute_interval < 1) return LITEVGGT_ERR_BAD_CONFIG;
   if (!(c.merge_ratio >= 0.0f && c.merge_ratio <= 1.0f)) return LITEVGGT_ERR_BAD_CONFIG;
   if (!(c.ga_keep_frac >= 0.0f && c.ga_keep_frac <= 1.0f)) return LITEVGGT_ERR_BAD_CONFIG;
-  if (c.qkv_dtype != 0) return LITEVGGT_ERR_BAD_CONFIG;
+  if (c.qkv_dtype != 0 && c.qkv_dtype != 1) return LITEVGGT_ERR_BAD_CONFIG;  // bf16 or E4M3 attention operands
   if (c.patch_px > 30) return LITEVGGT_ERR_BAD_CONFIG;  // a patch and its two halo columns share a warp in the Grad map
   Sizes z;
   z.frames = c.frames; z.grid_h = c.grid_h; z.grid_w = c.grid_w; z.n_special = c.n_special;
@@ -297,6 +297,10 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   const size_t state_bytes = attention_state_bytes(z.n_merged, z.dim, z.heads, &ml_off);
   const size_t o_state = c.take<uint8_t>((long long)state_bytes);
   const size_t o_kmax = c.take<float>((long long)z.frames * z.heads);
+  const bool fp8 = cfg->qkv_dtype == 1;
+  const long long m_pad = round_up(z.n_merged, 128);
+  const size_t o_q8 = c.take<uint8_t>(fp8 ? z.n_merged * z.dim : 0), o_k8 = c.take<uint8_t>(fp8 ? z.n_merged * z.dim : 0);
+  const size_t o_v8 = c.take<uint8_t>(fp8 ? m_pad * z.dim : 0), o_amax = c.take<float>(48);
   const size_t o_status = c.take<uint32_t>(4);
   Workspace& ws = ctx->ws;
   if (cudaMalloc(&ws.base, c.off) != cudaSuccess) {
@@ -326,6 +330,12 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
     ws.attn_ml_state = reinterpret_cast<float*>(ws.base + o_state + ml_off);
   }
   ws.attn_kmax = reinterpret_cast<float*>(ws.base + o_kmax);
+  if (fp8) {
+    ws.q8 = ws.base + o_q8;
+    ws.k8 = ws.base + o_k8;
+    ws.v8t = ws.base + o_v8;
+    ws.qkv_amax = reinterpret_cast<float*>(ws.base + o_amax);
+  }
   ws.status = reinterpret_cast<uint32_t*>(ws.base + o_status);
   if (cudaMemset(ws.base + o_var, 0, o_src - o_var) != cudaSuccess ||
       cudaMemset(ws.status, 0, 16) != cudaSuccess) {
@@ -541,9 +551,14 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
     e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d, static_cast<const __nv_bfloat16*>(w_qkv),
                       3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.qkv, s, &n);
   }
+  if (e == cudaSuccess && ctx->cfg.qkv_dtype == 1) {
+    StepTimer t(ctx, 14, s);
+    e = launch_qkv_quantize(ctx, ctx->ws.qkv, m, s, &n);
+  }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 7, s);
-    e = launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
+    e = ctx->cfg.qkv_dtype == 1 ? launch_flash_attention_fp8(ctx, m, ctx->ws.attn_o, s, &n)
+                                : launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 8, s);
@@ -594,9 +609,14 @@ litevggt_status litevggt_global_attn_ext(litevggt_ctx* ctx, const litevggt_plan*
                         static_cast<const __nv_bfloat16*>(ext->k_norm_beta), ext->norm_eps, ext->rope != 0,
                         ext->rope_base, s, &n);
   }
+  if (e == cudaSuccess && ctx->cfg.qkv_dtype == 1) {
+    StepTimer t(ctx, 14, s);
+    e = launch_qkv_quantize(ctx, ctx->ws.qkv, m, s, &n);
+  }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 7, s);
-    e = launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
+    e = ctx->cfg.qkv_dtype == 1 ? launch_flash_attention_fp8(ctx, m, ctx->ws.attn_o, s, &n)
+                                : launch_flash_attention(ctx, ctx->ws.qkv, m, 1, ctx->ws.attn_o, s, &n);
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 8, s);
@@ -905,6 +925,12 @@ litevggt_status litevggt_debug_buffer(litevggt_ctx* ctx, int which, void** dev_p
   } else if (which == 1) {
     *dev_ptr = ctx->ws.attn_o;
     if (bytes) *bytes = (size_t)z.n_merged * z.dim * 2;
+  } else if (which >= 2 && which <= 5 && ctx->cfg.qkv_dtype == 1) {
+    const size_t mp = (size_t)round_up(z.n_merged, 128);
+    void* ptrs[4] = {ctx->ws.q8, ctx->ws.k8, ctx->ws.v8t, ctx->ws.qkv_amax};
+    const size_t sizes[4] = {(size_t)z.n_merged * z.dim, (size_t)z.n_merged * z.dim, mp * z.dim, 48 * sizeof(float)};
+    *dev_ptr = ptrs[which - 2];
+    if (bytes) *bytes = sizes[which - 2];
   } else {
     return LITEVGGT_ERR_SHAPE;
   }

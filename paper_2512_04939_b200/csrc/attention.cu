@@ -558,6 +558,378 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// E4M3 variant (qkv_dtype = 1).  Same CTA shape, warp roles, barriers and tensor-memory map as the
+// bf16 kernel above; what differs:
+//   * Q, K and V arrive as E4M3 bytes with one scale per (tensor, head); both products run as
+//     kind::f8f6f4 (K = 32 per instruction: two instructions per step and product instead of four);
+//   * K tiles are 128 keys x 64 bytes (64-byte swizzle); V comes transposed, 64 channel rows x 128
+//     key bytes per tile, K-major like K, followed in shared memory by 16 rows of which the first
+//     holds 1.0 in every byte: as rows 64..79 of the B operand they make accumulator column 64 the sum
+//     of the very E4M3 probabilities that multiply V;
+//   * the probabilities are rounded to E4M3, whose values reach from 2^-9 to 448 only, so they must
+//     sit at the top of that range: every row runs the online form with the reference kept 8 below
+//     the running row maximum (the largest probability of a row is 2^8 when the reference is set
+//     and may grow to 2^8.75 before the row is rescaled), which leaves 17 binades below the row
+//     maximum before a probability is rounded to zero;
+//   * scores are multiplied by scale_q scale_k, the output by scale_v, in fp32.
+constexpr int kFa8KTileBytes = 128 * 64;           // 128 keys x 64 channel bytes
+constexpr int kFa8VTileBytes = 64 * 128;           // 64 channels x 128 key bytes
+constexpr int kFa8VStageBytes = kFa8VTileBytes + 16 * 128;  // + the ones rows
+constexpr uint32_t kFa8ColQ = 416;                 // Q_0, Q_1: 16 columns of 4 bytes each
+constexpr float kFa8Headroom = 8.0f;               // the row maximum maps to 2^8 of E4M3's 448
+constexpr int kFa8SmemBytes = kFaStages * (kFa8KTileBytes + kFa8VStageBytes) + (int)sizeof(FaExchange) + 512 + 1024;
+
+template <bool kFirst, bool kLast>
+__global__ void __launch_bounds__(kFaThreads, 1)
+flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __grid_constant__ CUtensorMap tmap_v8t,
+                           const uint8_t* __restrict__ q8, const float* __restrict__ amax, __nv_bfloat16* __restrict__ o,
+                           float* __restrict__ o_state, float* __restrict__ ml_state, int seq_len, int dim, int tile_begin,
+                           int tile_end, uint32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_k = smem;
+  uint8_t* smem_v = smem_k + kFaStages * kFa8KTileBytes;
+  FaExchange* xchg = reinterpret_cast<FaExchange*>(smem_v + kFaStages * kFa8VStageBytes);
+  FaBarriers* bars = reinterpret_cast<FaBarriers*>(xchg + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * 256;
+  const int head = blockIdx.y;
+  const int n_kv = tile_end - tile_begin;
+  const int n_steps = 2 * n_kv;
+  constexpr bool first_chunk = kFirst;
+  constexpr bool last_chunk = kLast;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->q_ready, kFaSoftmaxWarps);
+    for (int s = 0; s < kFaStages; ++s) {
+      mbar_init(&bars->k_full[s], 1);
+      mbar_init(&bars->k_empty[s], 2);
+      mbar_init(&bars->v_full[s], 1);
+      mbar_init(&bars->v_empty[s], 2);
+    }
+    for (int t = 0; t < 2; ++t) {
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(&bars->s_full[t][h], 1);
+        mbar_init(&bars->p_ready[t][h], 8);
+      }
+      mbar_init(&bars->pv_done[t], 1);
+      mbar_init(&bars->o_done[t], 1);
+    }
+    mbar_init(&bars->teardown[0], 1);
+    mbar_init(&bars->teardown[1], 1);
+    bars->abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmap_k8);
+    tma_prefetch_desc(&tmap_v8t);
+  }
+  // the ones rows behind every V stage: 128 bytes of E4M3 1.0 (0x38), then 15 rows of zeros (a row
+  // of equal bytes looks the same under the swizzle)
+  for (int i = threadIdx.x; i < kFaStages * 16 * 128 / 16; i += kFaThreads) {
+    const int stage = i / 128, piece = i % 128;  // 128 16-byte pieces per stage
+    const uint32_t fill = piece < 8 ? 0x38383838u : 0u;
+    reinterpret_cast<uint4*>(smem_v + stage * kFa8VStageBytes + kFa8VTileBytes)[piece] = make_uint4(fill, fill, fill, fill);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 16) {
+    tmem_alloc(&bars->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  const WaitCtl ctl{&bars->abort_flag, status};
+
+  if (warp == 17) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      uint32_t k_issued = 0, v_issued = 0;
+      for (int j = 0; j < n_kv; ++j) {
+        const int stage = j % kFaStages;
+        const uint32_t phase = (uint32_t)(j / kFaStages) & 1u;
+        if (!mbar_wait(&bars->k_empty[stage], phase ^ 1u, ctl)) break;
+        mbar_expect_tx(&bars->k_full[stage], kFa8KTileBytes);
+        tma_load_2d(smem_k + stage * kFa8KTileBytes, &tmap_k8, &bars->k_full[stage], head * 64, (tile_begin + j) * 128);
+        ++k_issued;
+        if (!mbar_wait(&bars->v_empty[stage], phase ^ 1u, ctl)) break;
+        mbar_expect_tx(&bars->v_full[stage], kFa8VTileBytes);
+        tma_load_2d(smem_v + stage * kFa8VStageBytes, &tmap_v8t, &bars->v_full[stage], (tile_begin + j) * 128, head * 64);
+        ++v_issued;
+      }
+      drain_ring(bars->k_full, k_issued, status);
+      drain_ring(bars->v_full, v_issued, status);
+    }
+  } else if (warp == 16 || warp == 18) {
+    // ------------------------------------------------------------------ MMA issuer of tile t
+    if (elect_one()) {
+      const int t = warp == 16 ? 0 : 1;
+      constexpr uint32_t idesc_qk = umma_idesc_e4m3(128, 64);
+      constexpr uint32_t idesc_pv = umma_idesc_e4m3(128, kFaOCols);
+      const uint32_t s_col = tmem_base + kFaColS + t * 128;
+      const uint32_t o_col = tmem_base + kFaColO + t * kFaOCols;
+      const uint32_t q_col = tmem_base + kFa8ColQ + t * 16;
+      // S_h = Q x K[64h .. 64h+63]^T: 64 rows of 64 bytes = 4096 bytes per half, 32 channels per instruction
+      auto issue_qk = [&](int h, int stage) {
+        const uint64_t b_desc = smem_desc_sw64(smem_u32(smem_k + stage * kFa8KTileBytes + h * 4096), 16, 512);
+#pragma unroll
+        for (int k = 0; k < 2; ++k) umma_ts_f8(s_col + h * 64, q_col + k * 8, b_desc + 2 * k, idesc_qk, k != 0 ? 1u : 0u);
+        umma_commit(&bars->s_full[t][h]);
+      };
+      bool ok = mbar_wait(&bars->q_ready, 0, ctl);
+      if (ok) ok = mbar_wait(&bars->k_full[0], 0, ctl);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        issue_qk(1, 0);
+        umma_commit(&bars->k_empty[0]);
+      }
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int j = 0; j < n_kv && ok; ++j) {
+        int next_stage = stage + 1;
+        uint32_t next_phase = phase;
+        if (next_stage == kFaStages) { next_stage = 0; next_phase ^= 1u; }
+        const bool last = j + 1 == n_kv;
+        if (!mbar_wait(&bars->v_full[stage], phase, ctl)) { ok = false; break; }
+        if (!last && !mbar_wait(&bars->k_full[next_stage], next_phase, ctl)) { ok = false; break; }
+        for (int h = 0; h < 2; ++h) {
+          if (!mbar_wait(&bars->p_ready[t][h], j & 1, ctl)) { ok = false; break; }
+          tc_fence_after();
+          // 64 keys of the transposed V tile: bytes [64h, 64h + 64) of every channel row, 32 keys per
+          // instruction; 8 tensor-memory columns of P each (keys 0-31 in columns [0,8) of the half,
+          // keys 32-63 in [32,40)); rows 64..79 of B are the ones rows behind the tile
+          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFa8VStageBytes + h * 64), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 2; ++k)
+            umma_ts_f8(o_col, s_col + h * 64 + k * 32, v_desc + 2 * k, idesc_pv, (j | h | k) != 0 ? 1u : 0u);
+          if (last) {
+            umma_commit(&bars->pv_done[t]);
+            if (h == 1) umma_commit(&bars->o_done[t]);
+          } else {
+            issue_qk(h, next_stage);
+          }
+        }
+        if (!ok) break;
+        umma_commit(&bars->v_empty[stage]);
+        if (!last) umma_commit(&bars->k_empty[next_stage]);
+        stage = next_stage;
+        phase = next_phase;
+      }
+      if (!ok) {
+        umma_commit(&bars->teardown[t]);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&bars->teardown[t], 0)) {
+          if (clock64() - t0 > kTimeoutCycles) break;
+        }
+      }
+    }
+  } else if (warp < kFaSoftmaxWarps) {
+    // ------------------------------------------------------------------ softmax warps
+    const int t = warp >> 3;
+    const int c = (warp >> 2) & 1;
+    const uint32_t quarter = warp & 3u;
+    const int barrier_id = 1 + t * 4 + (int)quarter;
+    const int row_in_tile = (int)quarter * 32 + lane;
+    const uint32_t lane_base = (quarter * 32u) << 16;
+    const int row_local = q0 + t * 128 + row_in_tile;
+    const bool row_live = row_local < seq_len;
+    const int row = row_local;
+    const uint32_t s_addr = tmem_base + lane_base + kFaColS + t * 128;
+    const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + c * 32;
+    const uint32_t l_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + 64;
+    {
+      // this thread's 32 channels (32 bytes) of its query row
+      uint32_t qreg[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) qreg[i] = 0u;
+      if (row_live) {
+        const uint4* src = reinterpret_cast<const uint4*>(q8 + (size_t)row * dim + head * 64 + c * 32);
+        const uint4 a = __ldg(src), b = __ldg(src + 1);
+        qreg[0] = a.x; qreg[1] = a.y; qreg[2] = a.z; qreg[3] = a.w;
+        qreg[4] = b.x; qreg[5] = b.y; qreg[6] = b.z; qreg[7] = b.w;
+      }
+      tmem_st8(tmem_base + lane_base + kFa8ColQ + t * 16 + c * 8, qreg);
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->q_ready);
+    }
+    // dequantisation: score = (q8 . k8) scale_q scale_k / sqrt(64), output = (P v8) scale_v / sum P
+    const float a_q = amax[head], a_k = amax[16 + head], a_v = amax[32 + head];
+    const float scale_q = (a_q > 0.0f ? a_q : 1.0f) / 448.0f, scale_k = (a_k > 0.0f ? a_k : 1.0f) / 448.0f;
+    const float scale_v = (a_v > 0.0f ? a_v : 1.0f) / 448.0f;
+    const float scale_log2e = 0.125f * 1.4426950408889634f * scale_q * scale_k;
+    const float2 scale2 = make_float2(scale_log2e, scale_log2e);
+    float m_ref = -INFINITY;
+    bool ok = true;
+    int pair_syncs = 0;
+    for (int n = 0; n < n_steps; ++n) {
+      const int j = n >> 1, h = n & 1;
+      if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t s[32];
+      tmem_ld32(s_addr + h * 64 + c * 32, s);
+      tmem_ld_wait();
+      const int valid = seq_len - (tile_begin * 2 + n) * 64 - c * 32;
+      if (valid < 32) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (i >= valid) s[i] = 0xff800000u;  // -inf
+      }
+      float mx[4];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t* sc = &s[g * 8];
+        mx[g] = fmax3(__uint_as_float(sc[0]), __uint_as_float(sc[1]), __uint_as_float(sc[2]));
+        mx[g] = fmax3(mx[g], __uint_as_float(sc[3]), __uint_as_float(sc[4]));
+        mx[g] = fmax3(mx[g], __uint_as_float(sc[5]), __uint_as_float(sc[6]));
+        mx[g] = fmaxf(mx[g], __uint_as_float(sc[7]));
+      }
+      const float mx_own = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
+      xchg->row_max[n & 1][t][c][row_in_tile] = mx_own;
+      pair_barrier(barrier_id);
+      ++pair_syncs;
+      const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
+      if (n == 0) {
+        m_ref = mx_scaled - kFa8Headroom;
+      } else {
+        const bool grow = mx_scaled > m_ref + kFa8Headroom + 0.75f;
+        if (__any_sync(0xffffffffu, grow ? 1 : 0)) {
+          const int jp = h == 1 ? j : j - 1;
+          const bool waited = jp + 1 < n_kv
+                                  ? mbar_wait_warp(&bars->s_full[t][h ^ 1], (uint32_t)(jp + 1) & 1u, ctl)
+                                  : mbar_wait_warp(&bars->pv_done[t], 0, ctl);
+          if (!waited) { ok = false; break; }
+          tc_fence_after();
+          const float m_new = grow ? mx_scaled - kFa8Headroom : m_ref;
+          const float alpha = fast_exp2(m_ref - m_new);
+          m_ref = m_new;
+          uint32_t acc[32];
+          tmem_ld32(o_addr, acc);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * alpha);
+          tmem_st32(o_addr, acc);
+          if (c == 1) {
+            uint32_t sum[16];
+            tmem_ld16(l_addr, sum);
+            tmem_ld_wait();
+            sum[0] = __float_as_uint(__uint_as_float(sum[0]) * alpha);
+            tmem_st16(l_addr, sum);
+          }
+        }
+      }
+      const float2 neg_m2 = make_float2(-m_ref, -m_ref);
+      uint32_t packed[8];  // 32 probabilities as E4M3 bytes
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[4 * i]), __uint_as_float(s[4 * i + 1])), scale2, neg_m2);
+        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[4 * i + 2]), __uint_as_float(s[4 * i + 3])), scale2, neg_m2);
+        packed[i] = pack_e4m3x4(fast_exp2(x0.x), fast_exp2(x0.y), fast_exp2(x1.x), fast_exp2(x1.y));
+      }
+      tmem_st8(s_addr + h * 64 + c * 32, packed);  // over the start of the columns just read
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
+    }
+    for (; pair_syncs < n_steps; ++pair_syncs) pair_barrier(barrier_id);
+    if (ok && mbar_wait_warp(&bars->o_done[t], 0, ctl)) {
+      tc_fence_after();
+      uint32_t acc[32], sum[16];
+      tmem_ld32(o_addr, acc);
+      tmem_ld16(l_addr, sum);
+      tmem_ld_wait();
+      if (row_live) {
+        float row_sum = __uint_as_float(sum[0]);
+        float* ml_mine = ml_state + ((size_t)row * (dim / 64) + head) * 4 + 2 * c;
+        if (!first_chunk) {
+          const float m_old = ml_mine[0], l_old = ml_mine[1];
+          float a_old = 1.0f, a_new = 1.0f;
+          if (m_old != m_ref) {
+            const float m_tot = fmaxf(m_old, m_ref);
+            a_old = fast_exp2(m_old - m_tot);
+            a_new = fast_exp2(m_ref - m_tot);
+            m_ref = m_tot;
+          }
+          const uint4* src = reinterpret_cast<const uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 v = src[i];
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              acc[4 * i + e] = __float_as_uint(fmaf(__uint_as_float(acc[4 * i + e]), a_new, __uint_as_float(w[e]) * a_old));
+          }
+          row_sum = fmaf(row_sum, a_new, l_old * a_old);
+        }
+        if (last_chunk) {
+          const float inv = scale_v / row_sum;
+          uint4* dst = reinterpret_cast<uint4*>(o + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(acc[q * 8 + 0]) * inv, __uint_as_float(acc[q * 8 + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(acc[q * 8 + 2]) * inv, __uint_as_float(acc[q * 8 + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(acc[q * 8 + 4]) * inv, __uint_as_float(acc[q * 8 + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(acc[q * 8 + 6]) * inv, __uint_as_float(acc[q * 8 + 7]) * inv);
+            dst[q] = w;
+          }
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(o_state + (size_t)row * dim + head * 64 + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+          ml_mine[0] = m_ref;
+          ml_mine[1] = row_sum;
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 16) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+cudaError_t launch_flash_attention_fp8(litevggt_ctx* ctx, long long m, __nv_bfloat16* o, cudaStream_t s, int* launches) {
+  if (m == 0) return cudaSuccess;
+  const int dim = ctx->sz.dim;
+  Workspace& ws = ctx->ws;
+  if (dim != 1024 || ws.q8 == nullptr) return cudaErrorInvalidValue;
+  const long long m_pad = round_up(m, 128);
+  CUtensorMap tmap_k, tmap_v;
+  if (!make_tmap_u8_2d(ctx->encode_tiled, &tmap_k, ws.k8, (uint64_t)dim, (uint64_t)m, (uint64_t)dim, 64, 128) ||
+      !make_tmap_u8_2d(ctx->encode_tiled, &tmap_v, ws.v8t, (uint64_t)m_pad, (uint64_t)dim, (uint64_t)m_pad, 128, 64))
+    return cudaErrorInvalidValue;
+  using Kernel = void (*)(const CUtensorMap, const CUtensorMap, const uint8_t*, const float*, __nv_bfloat16*, float*,
+                          float*, int, int, int, int, uint32_t*);
+  const Kernel kernels[2][2] = {{flash_attention_fp8_kernel<false, false>, flash_attention_fp8_kernel<false, true>},
+                                {flash_attention_fp8_kernel<true, false>, flash_attention_fp8_kernel<true, true>}};
+  static std::atomic<unsigned long long> smem_set[2][2];
+  for (int a = 0; a < 2; ++a)
+    for (int b = 0; b < 2; ++b) {
+      cudaError_t e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(kernels[a][b]), kFa8SmemBytes, smem_set[a][b]);
+      if (e != cudaSuccess) return e;
+    }
+  const dim3 grid((unsigned)((m + 255) / 256), (unsigned)ctx->sz.heads, 1);
+  const int n_tiles = (int)((m + 127) / 128);
+  const int n_chunks = (n_tiles + kFaChunkTiles - 1) / kFaChunkTiles;
+  const int per_chunk = (n_tiles + n_chunks - 1) / n_chunks;
+  if (n_chunks > 1 && (ws.attn_o_state == nullptr || ws.attn_ml_state == nullptr)) return cudaErrorInvalidValue;
+  for (int begin = 0; begin < n_tiles; begin += per_chunk) {
+    const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
+    kernels[begin == 0][end == n_tiles]<<<grid, kFaThreads, kFa8SmemBytes, s>>>(
+        tmap_k, tmap_v, ws.q8, ws.qkv_amax, o, ws.attn_o_state, ws.attn_ml_state, (int)m, dim, begin, end, ws.status);
+    ++*launches;
+  }
+  return cudaGetLastError();
+}
+
 // max_k |k|^2 per (sequence, head), for the Cauchy-Schwarz bound on a row's scores.  Warp per key
 // row: the 128 16-byte pieces of a K row go to the lanes in four passes, eight neighbouring lanes
 // share a head.  Non-negative floats order like their bit patterns, so the maximum is an integer

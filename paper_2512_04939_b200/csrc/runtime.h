@@ -69,6 +69,11 @@ struct Workspace {
   float* attn_o_state = nullptr;   // [M, D] running output between key chunks (long sequences only)
   float* attn_ml_state = nullptr;  // [M, heads, 4] reference maximum and partial row sums
   float* attn_kmax = nullptr;      // [max(frames, 1), heads] largest |k|^2 per sequence and head
+  // E4M3 variant of the attention operands (qkv_dtype = 1)
+  uint8_t* q8 = nullptr;           // [M, D] bytes
+  uint8_t* k8 = nullptr;           // [M, D] bytes
+  uint8_t* v8t = nullptr;          // [D, round_up(M, 128)] bytes: V transposed, head-major rows
+  float* qkv_amax = nullptr;       // [3, heads] largest magnitude of Q, K, V per head
   // whole-layer-from-host staging
   __nv_bfloat16* stage_x = nullptr;   // [N, D]
   __nv_bfloat16* stage_xm = nullptr;  // [M, D]
@@ -86,7 +91,7 @@ struct Workspace {
 namespace lv {
 // Device-time stopwatches, one per step of the path: CUDA event pairs recorded on the
 // launching stream around the step's kernels, kept in a small ring per step.
-constexpr int kNumTimers = 14;
+constexpr int kNumTimers = 15;
 constexpr int kTimerSlots = 64;
 struct Timers {
   cudaEvent_t start[kNumTimers][kTimerSlots];
@@ -152,6 +157,8 @@ bool resolve_encode_tiled(void** fn);
 // 128-byte swizzle, zero fill outside the tensor.
 bool make_tmap_bf16_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
                        uint64_t pitch_elems, uint32_t box_inner, uint32_t box_outer);
+bool make_tmap_u8_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer,
+                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer);
 
 // scoring.cu
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches);
@@ -200,5 +207,9 @@ cudaError_t launch_qk_embed(const litevggt_ctx* ctx, __nv_bfloat16* qkv, const i
 cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long seq_len, int n_seq,
                                    __nv_bfloat16* o, cudaStream_t s, int* launches);
 size_t attention_state_bytes(long long m, int dim, int heads, size_t* ml_offset);
+// E4M3 variant: per-head amax of Q, K, V and their quantised copies (fp8_quant.cu), then the
+// attention core on those (attention.cu); one sequence of m rows
+cudaError_t launch_qkv_quantize(litevggt_ctx* ctx, const __nv_bfloat16* qkv, long long m, cudaStream_t s, int* launches);
+cudaError_t launch_flash_attention_fp8(litevggt_ctx* ctx, long long m, __nv_bfloat16* o, cudaStream_t s, int* launches);
 
 }  // namespace lv

@@ -679,3 +679,78 @@ def test_abi_misuse_returns_error_codes(lib):
     ctx.poll()  # flag was cleared
     p2.destroy(); plan.destroy()
     other.close(); ctx.close()
+
+
+# ------------------------------------------------------------------ E4M3 variant of the attention operands
+# Tolerances of the FP8 variant.  The quantised operands are judged bit for bit against the
+# oracle's quantiser (same scales, same codes).  The attention core is then judged on the GPU's own
+# quantised operands, dequantised, so that what remains is (a) the rounding of the probabilities to
+# E4M3 - relative error up to 2^-4, independent from key to key, over the sum of the same rounded
+# values: sum_i d_i p_i (v_i - o) / sum_i p_i with |d_i| <= 2^-4, i.e. at most 6.25 % of the spread
+# of the values a row attends to and 1/sqrt(3 n_eff) of that when n_eff keys share the mass - and
+# (b) the bf16 rounding of the output.  Nearly uniform rows (stock weights) therefore meet the bf16
+# bound plus FP8_FLAT_NOISE; rows held by a handful of keys get FP8_PEAKED_NOISE.
+FP8_FLAT_NOISE = 8e-3
+FP8_PEAKED_NOISE = 8e-2
+
+
+def _e4m3_decode(codes):
+    vals = np.concatenate([O.e4m3_values(), [np.nan]])
+    c = codes.cpu().numpy()
+    return np.where(c & 0x80, -1.0, 1.0) * vals[c & 0x7f]
+
+
+@pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
+def test_fp8_attention_variant(lib, wl):
+    _, tok = _inputs(wl)
+    _, ref = _oracle_plan(wl)
+    m = ref["sizes"]["M"]
+    xm = torch.from_numpy(O.merge(to_f64(tok), ref["dst_of"], m).astype(np.float32)).to(torch.bfloat16)
+    w_qkv, b_qkv, w_o, b_o = make_attention_weights(wl, 0)
+    w_big = (w_qkv.float() * 3.0).to(torch.bfloat16)
+    ctx = _ctx(lib, wl, qkv_dtype=1)
+    for tag, wq, noise in (("stock", w_qkv, FP8_FLAT_NOISE), ("3x", w_big, FP8_PEAKED_NOISE)):
+        y = ctx.global_attn(xm.cuda(), wq.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
+        ctx.poll()
+        qkv = to_f64(ctx.debug_buffer(0))   # the bf16 projection, as the bf16 path produces it
+        f8 = ctx.debug_fp8_buffers()
+        # quantisation: scales and codes equal the oracle's on the GPU's own projection
+        deq_ref, codes_ref, scales_ref = O.quantize_qkv_e4m3(qkv, heads=16)
+        amax = f8["amax"].cpu().numpy()
+        assert np.array_equal(amax / np.float32(448.0), scales_ref), "per-head scales"
+        d = 1024
+        got_codes = np.concatenate([f8["q8"].cpu().numpy(), f8["k8"].cpu().numpy(),
+                                    f8["v8t"].cpu().numpy()[:, :m].T], axis=1)
+        nonzero = (codes_ref & 0x7f) != 0  # the sign bit of a zero is free
+        assert np.array_equal(got_codes[nonzero], codes_ref[nonzero]) and np.all((got_codes[~nonzero] & 0x7f) == 0)
+        assert np.all(f8["v8t"].cpu().numpy()[:, m:] == 0), "padded keys must be zero"
+        # the core on the dequantised operands
+        ref_o = O.attention_core(deq_ref, heads=16)
+        o = to_f64(ctx.debug_buffer(1))
+        check_bf16(f"fp8 {wl.name}/{tag}: attention core", o, ref_o, noise=noise)
+        # against the unquantised core: what the 8-bit operands cost (reported, loosely bounded)
+        ref_o_bf16 = O.attention_core(qkv, heads=16)
+        report(f"fp8 {wl.name}/{tag}: attention core vs unquantised operands", err_over_rms=rel_err(o, ref_o_bf16))
+        assert rel_err(o, ref_o_bf16) < (0.1 if tag == "stock" else 1.0)
+        check_bf16(f"fp8 {wl.name}/{tag}: output projection", to_f64(y), O.linear(o, to_f64(w_o), to_f64(b_o)))
+    ctx.close()
+
+
+def test_fp8_attention_variant_with_peaked_softmax(lib):
+    """The E4M3 variant on the near-duplicate groups: every key tile matters, and a dropped tile on
+    the oracle's side is far outside the FP8 tolerance too."""
+    ctx = lib.LiteVGGT(2, 22, 33, 0.0, qkv_dtype=1)
+    m = ctx.n_merged
+    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, 31 + m, groups=97, sharpness=4.0)
+    ctx.global_attn(x.cuda(), w_qkv.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
+    ctx.poll()
+    deq, _, _ = O.quantize_qkv_e4m3(to_f64(ctx.debug_buffer(0)), heads=16)
+    ref_o = O.attention_core(deq, heads=16)
+    o = to_f64(ctx.debug_buffer(1))
+    check_bf16("fp8 peaked: attention core", o, ref_o, noise=FP8_PEAKED_NOISE)
+    keep = np.ones(m, bool)
+    keep[256:384] = False
+    rows = np.flatnonzero(keep)[:200]
+    ref_short = O.attention_core(deq[keep], heads=16, rows=np.arange(200))
+    assert rel_err(o[rows], ref_short) > 4 * (bf16_bound(ref_o) + FP8_PEAKED_NOISE)
+    ctx.close()
