@@ -126,7 +126,7 @@ class ClockSampler:
 #     partition, merge, unmerge) on a sub-sequence of `linear_frames` frames, x F / linear_frames
 #     (a float64 copy of the whole token matrix is 8.5 GB at 1000 frames);
 #   * selection + index build at full size (on seeded similarities: its cost does not depend on them).
-CPU_SAMPLE = dict(match_rows=1024, attn_rows=128, attn_heads=2, proj_rows=4096, linear_frames=64)
+CPU_SAMPLE = dict(match_rows=2048, attn_rows=256, attn_heads=4, proj_rows=8192, linear_frames=64)
 REF_SAMPLE = dict(match_rows=256, attn_rows=64, attn_heads=1, proj_rows=1024, linear_frames=16)
 
 
@@ -448,6 +448,25 @@ def run_ours(args, wl):
     stats_clocks = stats_sampler.stop() if rank == 0 else None
     stats_mhz = stats_clocks["sm_mhz"] if stats_clocks else None
 
+    # ---- the E4M3 variant of the attention operands, beside bf16 (same rows, same weights)
+    fp8 = None
+    if not args.no_fp8:
+        ctx8 = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, device=local, qkv_dtype=1)
+        ctx8.global_attn(xm, *weights[0], out=ym)
+        ctx8.poll()
+        ctx8.timers_reset()
+        for i in range(attn_reps):
+            ctx8.global_attn(xm, *weights[i % len(weights)], out=ym)
+        ctx8.poll()
+        s8 = ctx8.timers_samples()
+        ctx8.close()
+        core, quant = float(np.median(s8["attention"])), float(np.median(s8["qkv_quantize"]))
+        fp8 = {"attention_core_ms_median": round(core, 3), "attention_core_ms_best": round(min(s8["attention"]), 3),
+               "quantize_ms_median": round(quant, 3), "samples": len(s8["attention"]),
+               "TFLOP/s": round(4.0 * m * m * d / (core * 1e-3) / 1e12, 1),
+               "note": "qkv_dtype = 1: Q, K, V and the probabilities in E4M3, both products kind::f8f6f4; flops counted "
+                       "as for bf16 (4 M^2 D); parity: tests/test_gpu_parity.py::test_fp8_attention_variant"}
+
     block = None
     if args.block:
         # One aggregator block (Sec. 3.1), pre-norm: x += frame_attn(LN x); x += MLP(LN x);
@@ -558,6 +577,7 @@ def run_ours(args, wl):
                           "(attention layer: 5 at this size), median and best; ms_x_mhz = median ms x median SM MHz of "
                           "that pass (%s MHz)" % (stats_mhz,),
         "cpu_baseline": cpu,
+        "fp8_qkv_variant": fp8,
     }
     if block is not None:
         line["aggregator_block"] = block
@@ -574,6 +594,7 @@ def main():
     ap.add_argument("--workload", default="C5", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the timing of the E4M3 variant of the attention operands")
     ap.add_argument("--block", action="store_true",
                     help="also time whole aggregator blocks (LayerNorm, frame-local attention, MLP around the "
                          "merged global layer) and add an \"aggregator_block\" object to the line")

@@ -301,3 +301,56 @@ def test_qk_norm_and_rope_on_sampled_rows(run):
     assert rel_err(got[:, 2048:], ref[:, 2048:]) <= bf16_bound(ref[:, 2048:]), "V is only projected"
     ref_y = O.linear(to_f64(ctx.debug_buffer(1)[rows_t]), to_f64(w_o), to_f64(b_o))
     assert rel_err(to_f64(y[rows_t]), ref_y) <= bf16_bound(ref_y), "output projection"
+
+
+@pytest.mark.parametrize("name", ["C3", "C5"])
+def test_fp8_attention_variant_on_sampled_rows(name):
+    """The E4M3 variant (qkv_dtype = 1) at the merged lengths of C3 and C5, on the near-duplicate
+    groups so that every key chunk matters: per-head scales and the quantised codes of sampled rows
+    bit for bit against the oracle's quantiser, and the attention core of sampled queries against
+    the oracle on the GPU's own operands, dequantised (tolerances as in the small-size test)."""
+    import paper_2512_04939_b200 as pkg
+    from test_gpu_parity import FP8_PEAKED_NOISE
+
+    wl = WORKLOADS[name]
+    ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio, qkv_dtype=1)
+    m = ctx.n_merged
+    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, wl.seed + 9, "cuda")
+    ctx.global_attn(x, w_qkv, b_qkv, w_o, b_o)
+    ctx.poll()
+    qkv_gpu, o_gpu = ctx.debug_buffer(0), ctx.debug_buffer(1)
+    f8 = ctx.debug_fp8_buffers()
+    # scales: the largest magnitude of every (tensor, head) slice, exactly
+    amax_ref = qkv_gpu.float().abs().reshape(m, 3, 16, 64).amax(dim=(0, 3))
+    assert torch.equal(f8["amax"], amax_ref)
+    scales = (f8["amax"].cpu().numpy() / np.float32(448.0)).astype(np.float32)
+    edges, _ = key_chunk_edges(m)
+    rng = np.random.default_rng(19)
+    rows = [0, 127, 128, m - 1] + list(rng.choice(m, 12, replace=False))
+    for e in edges:
+        rows += [e - 1, e]
+    rows = np.unique(np.asarray(rows, dtype=np.int64))
+    rows_t = torch.from_numpy(rows).cuda()
+    # codes of the sampled rows (Q, K row-major; V from the transposed copy)
+    part = to_f64(qkv_gpu[rows_t])
+    per_elem = np.repeat(scales.reshape(48), 64)[None, :]
+    codes_ref, _ = O.quantize_e4m3(part, np.broadcast_to(per_elem, part.shape))
+    got = np.concatenate([f8["q8"][rows_t].cpu().numpy(), f8["k8"][rows_t].cpu().numpy(),
+                          f8["v8t"][:, rows_t].cpu().numpy().T], axis=1)
+    nonzero = (codes_ref & 0x7f) != 0
+    assert np.array_equal(got[nonzero], codes_ref[nonzero]) and np.all((got[~nonzero] & 0x7f) == 0)
+    assert torch.all(f8["v8t"][:, m:] == 0)
+    vals = np.concatenate([O.e4m3_values(), [np.nan]])
+    decode = lambda c: np.where(c & 0x80, -1.0, 1.0) * vals[c & 0x7f]
+    o_rows = to_f64(o_gpu[rows_t])
+    for head in (0, 9, 15):
+        sl = slice(64 * head, 64 * head + 64)
+        q = decode(f8["q8"][:, sl].cpu().numpy()) * scales[0, head]
+        k = decode(f8["k8"][:, sl].cpu().numpy()) * scales[1, head]
+        v = decode(f8["v8t"][sl, :m].cpu().numpy().T) * scales[2, head]
+        ref_o = O.attention_core(np.concatenate([q, k, v], axis=1), heads=1, rows=rows)
+        check_bf16(f"fp8 {name}: attention core, peaked softmax, head {head}", o_rows[:, sl], ref_o, noise=FP8_PEAKED_NOISE,
+                   sampled=True)
+    ctx.close()
+    del x, f8
+    torch.cuda.empty_cache()
