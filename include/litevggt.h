@@ -281,7 +281,9 @@ litevggt_status litevggt_plan_import(litevggt_ctx* ctx, const int32_t* dst_of, l
 litevggt_status litevggt_plan_destroy(litevggt_plan* plan);
 
 /* Pointer to an internal device buffer of the last litevggt_global_attn call (tests):
- * which = 0: qkv bf16 [M,3D];  which = 1: attention output o bf16 [M,D];  with qkv_dtype = 1 also
+ * which = 0: qkv bf16 [M,3D], whose K third is stored multiplied by the softmax scale in base-2
+ * units, 1/sqrt(64) log2(e), rounded once (the attention kernels take 2^(q . k) as it comes from the
+ * tensor core);  which = 1: attention output o bf16 [M,D];  with qkv_dtype = 1 also
  * 2: Q as E4M3 bytes [M,D];  3: K likewise;  4: V transposed, bytes [D, round_up(M,128)] (row =
  * head * 64 + channel, column = key, zero beyond M);  5: float [3, heads], the largest magnitude of
  * Q, K, V per head (scale = amax / 448). */

@@ -548,8 +548,9 @@ litevggt_status litevggt_global_attn(litevggt_ctx* ctx, const void* x_merged, in
   cudaError_t e;
   {
     StepTimer t(ctx, 6, s);
-    e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d, static_cast<const __nv_bfloat16*>(w_qkv),
-                      3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.qkv, s, &n);
+    e = launch_linear_scaled(ctx, static_cast<const __nv_bfloat16*>(x_merged), m, d,
+                             static_cast<const __nv_bfloat16*>(w_qkv), 3 * d, static_cast<const __nv_bfloat16*>(b_qkv), d,
+                             2 * d, kKeyScaleLog2e, ctx->ws.qkv, s, &n);
   }
   if (e == cudaSuccess && ctx->cfg.qkv_dtype == 1) {
     StepTimer t(ctx, 14, s);
@@ -660,8 +661,9 @@ litevggt_status litevggt_frame_attn(litevggt_ctx* ctx, const void* x, const void
   cudaError_t e;
   {
     StepTimer t(ctx, 11, s);
-    e = launch_linear(ctx, static_cast<const __nv_bfloat16*>(x), z.n_tokens, d, static_cast<const __nv_bfloat16*>(w_qkv),
-                      3 * d, static_cast<const __nv_bfloat16*>(b_qkv), ctx->ws.blk_qkv, s, &n);
+    e = launch_linear_scaled(ctx, static_cast<const __nv_bfloat16*>(x), z.n_tokens, d,
+                             static_cast<const __nv_bfloat16*>(w_qkv), 3 * d, static_cast<const __nv_bfloat16*>(b_qkv), d,
+                             2 * d, kKeyScaleLog2e, ctx->ws.blk_qkv, s, &n);
     if (e == cudaSuccess) e = launch_flash_attention(ctx, ctx->ws.blk_qkv, z.tokens_frame, z.frames, ctx->ws.blk_o, s, &n);
     if (e == cudaSuccess)
       e = launch_linear_mlp(ctx, ctx->ws.blk_o, z.n_tokens, d, static_cast<const __nv_bfloat16*>(w_o), d,

@@ -41,8 +41,9 @@
 // evaluated on the FMA pipes instead: round-to-nearest split x = n + f, |f| <= 1/2, a cubic
 // for 2^f (relative error 7.5e-5, far below the bf16 rounding of P) and n added into the
 // exponent field.  The share is a build-time constant, kFaPolyPairs of the 16 pairs of scores a
-// thread handles per step; 6 measured best (4 warps per scheduler on register data alone: 182
-// clocks per 32 scores against 257 with the special-function unit only; 8 pairs: 220).
+// thread handles per step; 7 measured best in the kernel (on register data alone, 4 warps per
+// scheduler: 6 pairs take 182 clocks per 32 scores against 257 with the special-function unit only,
+// 8 pairs 220).
 // Shared memory: K ring, V ring, and behind the V ring a block of the same size that holds the
 // ones column of the P V operand for every ring position (see the kernel).
 //
@@ -61,13 +62,15 @@
 // Softmax reference.  Any per-row constant m may be subtracted from the scores before the
 // exponential: the division by the row sum removes it again.  It only has to keep 2^(s - m)
 // inside the range of bf16 / fp32, it does not have to be the row maximum.  By Cauchy-Schwarz
-// every score of a row is at most B = |q| max_k |k| (times the softmax scale, in base-2 units), so
+// every score of a row is at most B = |q| max_k |k| (K carrying the softmax scale: base-2 units), so
 // with m = B all exponents lie in [-2B, 0]; while 2B stays well inside the exponent range of
 // fp32 nothing underflows, every probability keeps its 8 significant bits and the fp32
 // accumulators their 24.  A small pass over K finds max_k |k|^2 per head before the sweep, each
 // softmax thread takes |q|^2 of its row while loading Q, and a warp pair whose rows all have
-// B <= kFaFixedRefLimit runs the sweep with that constant: no row maximum, no exchange between
-// the two threads of a row, no rescaling.  Rows with larger B (scores that could span more than
+// B <= kFaFixedRefLimit runs the sweep with a constant reference (in fact with none: the constant
+// cancels, see the kernel): no row maximum, no exchange between the two threads of a row, no
+// rescaling, and - the softmax scale 1/sqrt(64) log2(e) arriving folded into K - no arithmetic
+// between the tensor core's scores and the exponential.  Rows with larger B (scores that could span more than
 // the exponent range allows) take the online form: base-2 softmax with a lazily updated reference
 // maximum, the running output rescaled only when a row maximum grows by more than 2^8 over the
 // reference (the threads then first wait until the tile's last P V has retired).  Both forms equal
@@ -97,7 +100,7 @@ constexpr int kFaChunkTiles = LV_FA_CHUNK_TILES;  // 65536 keys: K and V of one 
 // Of the 16 pairs of scores a thread handles per step, this many take the polynomial exponential
 // (fixed-reference form only, where every argument lies in [-2 * kFaFixedRefLimit, 0]).
 #ifndef LV_FA_POLY_PAIRS
-#define LV_FA_POLY_PAIRS 6
+#define LV_FA_POLY_PAIRS 7
 #endif
 constexpr int kFaPolyPairs = LV_FA_POLY_PAIRS;
 
@@ -175,6 +178,23 @@ __device__ __forceinline__ void softmax_chunk(const uint32_t (&s)[32], float2 sc
   }
 }
 
+// The same for scores that arrive already scaled, with no reference to subtract: p = 2^s.
+template <int kPoly>
+__device__ __forceinline__ void exp2_chunk(const uint32_t (&s)[32], uint32_t (&packed)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float2 x = make_float2(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+    float2 p;
+    if (i < kPoly) {
+      p = poly_exp2_pair(x);
+    } else {
+      p.x = fast_exp2(x.x);
+      p.y = fast_exp2(x.y);
+    }
+    packed[i] = pack_bf16(p.x, p.y);
+  }
+}
+
 __device__ __forceinline__ void pair_barrier(int id) {  // the two warps of one (tile, lane quarter)
   asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
 }
@@ -185,7 +205,7 @@ __global__ void __launch_bounds__(kFaThreads, 1)
 flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_bfloat16* __restrict__ qkv,
                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_state, float* __restrict__ ml_state,
                        const float* __restrict__ k_norm2_max, int seq_len, int dim, int tile_begin, int tile_end,
-                       float scale_log2e, uint32_t* status) {
+                       uint32_t* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_k = smem;
@@ -356,8 +376,9 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
     const uint32_t o_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + c * 32;
     const uint32_t l_addr = tmem_base + lane_base + kFaColO + t * kFaOCols + 64;  // row sum column (+15 unused)
     float q_norm2 = 0.0f;  // |q|^2 of the whole row, summed in the same order by both of its threads
+    bool fixed_ref;
     {
-      // this thread's half (32 channels) of its query row goes to tensor memory as it is
+      // this thread's half (32 channels) of its query row goes to tensor memory
       uint32_t qreg[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) qreg[i] = 0u;
@@ -377,24 +398,26 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           }
         }
       }
+      // Cauchy-Schwarz bound on this row's scores (K carries the softmax scale, so the scores are in
+      // base-2 units already); both threads of a row hold the same value, and both warps of a pair
+      // vote over the same 32 rows, so they agree on the form they run
+      const float score_bound = sqrtf(q_norm2 * k_norm2_max[blockIdx.z * gridDim.y + head]);
+      fixed_ref = __all_sync(0xffffffffu, score_bound <= kFaFixedRefLimit ? 1 : 0) != 0;
       tmem_st16(tmem_base + lane_base + kFaColQ + t * 32 + c * 16, qreg);
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->q_ready);
     }
-    const float2 scale2 = make_float2(scale_log2e, scale_log2e);
-    // Cauchy-Schwarz bound on this row's scores in base-2 units; both threads of a row hold the same
-    // value, and both warps of a pair vote over the same 32 rows, so they agree on the form they run
-    const float score_bound = sqrtf(q_norm2 * k_norm2_max[blockIdx.z * gridDim.y + head]) * scale_log2e;
-    const bool fixed_ref = __all_sync(0xffffffffu, score_bound <= kFaFixedRefLimit ? 1 : 0) != 0;
-    float m_ref = -INFINITY;  // reference, in log2 units (score * scale * log2 e)
+    float m_ref = -INFINITY;  // reference, in the scores' own (base-2) units
     bool ok = true;
     int pair_syncs = 0;  // both warps of a pair must pass the same number of pair barriers
     if (fixed_ref) {
-      // ---- fixed reference: every exponent lies in [-2 * score_bound, 0]
-      m_ref = score_bound;
-      const float2 neg_m2 = make_float2(-m_ref, -m_ref);
+      // ---- fixed reference.  The scores all lie inside [-score_bound, score_bound]; the constant
+      // 2^-score_bound that would bring the exponents to [-2 score_bound, 0] cancels between numerator
+      // and row sum, so it is not applied: reference 0, and the scores go into the exponential as
+      // they come out of the tensor core.
+      m_ref = 0.0f;
       pair_syncs = n_steps;  // this form has no pair barriers
       for (int n = 0; n < n_steps; ++n) {
         const int j = n >> 1, h = n & 1;
@@ -409,9 +432,9 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
 #pragma unroll
           for (int i = 0; i < 32; ++i)
             if (i >= valid) s[i] = 0xff800000u;  // -inf: probability 0 (the polynomial cannot take it)
-          softmax_chunk<0>(s, scale2, neg_m2, packed);
+          exp2_chunk<0>(s, packed);
         } else {
-          softmax_chunk<kFaPolyPairs>(s, scale2, neg_m2, packed);
+          exp2_chunk<kFaPolyPairs>(s, packed);
         }
         tmem_st16(s_addr + h * 64 + c * 32, packed);  // over the start of the columns just read
         tmem_st_wait();
@@ -448,7 +471,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       xchg->row_max[n & 1][t][c][row_in_tile] = mx_own;
       pair_barrier(barrier_id);
       ++pair_syncs;
-      const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
+      const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]);
       if (n == 0) {
         m_ref = mx_scaled;
       } else {
@@ -483,7 +506,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       }
       const float2 neg_m2 = make_float2(-m_ref, -m_ref);
       uint32_t packed[16];
-      softmax_chunk<0>(s, scale2, neg_m2, packed);
+      softmax_chunk<0>(s, make_float2(1.0f, 1.0f), neg_m2, packed);
       tmem_st16(s_addr + h * 64 + c * 32, packed);  // over the start of the columns just read
       tmem_st_wait();
       tc_fence_before();
@@ -572,7 +595,8 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
 //     the running row maximum (the largest probability of a row is 2^8 when the reference is set
 //     and may grow to 2^8.75 before the row is rescaled), which leaves 17 binades below the row
 //     maximum before a probability is rounded to zero;
-//   * scores are multiplied by scale_q scale_k, the output by scale_v, in fp32.
+//   * scores are multiplied by scale_q scale_k (K arrives with the softmax scale folded in, which its
+//     per-head scale absorbs), the output by scale_v, in fp32.
 constexpr int kFa8KTileBytes = 128 * 64;           // 128 keys x 64 channel bytes
 constexpr int kFa8VTileBytes = 64 * 128;           // 64 channels x 128 key bytes
 constexpr int kFa8VStageBytes = kFa8VTileBytes + 16 * 128;  // + the ones rows
@@ -760,7 +784,7 @@ flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __
     const float a_q = amax[head], a_k = amax[16 + head], a_v = amax[32 + head];
     const float scale_q = (a_q > 0.0f ? a_q : 1.0f) / 448.0f, scale_k = (a_k > 0.0f ? a_k : 1.0f) / 448.0f;
     const float scale_v = (a_v > 0.0f ? a_v : 1.0f) / 448.0f;
-    const float scale_log2e = 0.125f * 1.4426950408889634f * scale_q * scale_k;
+    const float scale_log2e = scale_q * scale_k;  // K was quantised with the softmax scale folded in
     const float2 scale2 = make_float2(scale_log2e, scale_log2e);
     float m_ref = -INFINITY;
     bool ok = true;
@@ -985,7 +1009,7 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap, qkv, (uint64_t)3 * dim, (uint64_t)rows, (uint64_t)3 * dim, 64, 128))
     return cudaErrorInvalidValue;
   using Kernel = void (*)(const CUtensorMap, const __nv_bfloat16*, __nv_bfloat16*, float*, float*, const float*, int,
-                          int, int, int, float, uint32_t*);
+                          int, int, int, uint32_t*);
   const Kernel kernels[2][2] = {{flash_attention_kernel<false, false>, flash_attention_kernel<false, true>},
                                 {flash_attention_kernel<true, false>, flash_attention_kernel<true, true>}};
   static std::atomic<unsigned long long> smem_set[2][2];
@@ -995,7 +1019,6 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
       if (e != cudaSuccess) return e;
     }
   const dim3 grid((unsigned)((seq_len + 255) / 256), (unsigned)ctx->sz.heads, (unsigned)n_seq);
-  const float scale_log2e = 0.125f * 1.4426950408889634f;
   // balanced chunks of at most kFaChunkTiles key tiles; more than one needs the state buffers (which
   // are sized for the single long sequence of the global layer)
   const int n_tiles = (int)((seq_len + 127) / 128);
@@ -1007,7 +1030,7 @@ cudaError_t launch_flash_attention(litevggt_ctx* ctx, const __nv_bfloat16* qkv, 
     const int end = begin + per_chunk < n_tiles ? begin + per_chunk : n_tiles;
     kernels[begin == 0][end == n_tiles]<<<grid, kFaThreads, kFaSmemBytes, s>>>(
         tmap, qkv, o, ctx->ws.attn_o_state, ctx->ws.attn_ml_state, ctx->ws.attn_kmax, (int)seq_len, dim, begin, end,
-        scale_log2e, ctx->ws.status);
+        ctx->ws.status);
     ++*launches;
   }
   return cudaGetLastError();

@@ -107,9 +107,10 @@ extern "C" litevggt_status litevggt_global_attn_static(const void* x_merged, int
   local.ws.status = status;
   local.ws.attn_kmax = reinterpret_cast<float*>(dev->scratch + 64);  // zeroed by the attention launcher
   int n = 0;
-  cudaError_t e = lv::launch_linear(&local, static_cast<const __nv_bfloat16*>(x_merged), m, kStaticDim,
-                                    static_cast<const __nv_bfloat16*>(w_qkv), 3 * kStaticDim,
-                                    static_cast<const __nv_bfloat16*>(b_qkv), qkv, s, &n);
+  cudaError_t e = lv::launch_linear_scaled(&local, static_cast<const __nv_bfloat16*>(x_merged), m, kStaticDim,
+                                           static_cast<const __nv_bfloat16*>(w_qkv), 3 * kStaticDim,
+                                           static_cast<const __nv_bfloat16*>(b_qkv), kStaticDim, 2 * kStaticDim,
+                                           lv::kKeyScaleLog2e, qkv, s, &n);
   if (e == cudaSuccess) e = lv::launch_flash_attention(&local, qkv, m, 1, o, s, &n);
   if (e == cudaSuccess)
     e = lv::launch_linear(&local, o, m, kStaticDim, static_cast<const __nv_bfloat16*>(w_o), kStaticDim,

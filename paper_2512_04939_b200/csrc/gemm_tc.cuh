@@ -280,11 +280,14 @@ struct LinearEpilogue {
   const __nv_bfloat16* bias;  // may be null
   int m_rows;
   int n_cols;
+  int scale_begin, scale_end;  // output columns [scale_begin, scale_end) are multiplied by `scale`
+  float scale;
 
   __device__ __forceinline__ void begin(State&, int) const {}
   __device__ __forceinline__ void finish(State&, int) const {}
   // 64 accumulator columns of one row -> 32 bf16 pairs
   __device__ __forceinline__ void transform(int, int col0, const uint32_t (&acc)[64], uint32_t (&packed)[32]) const {
+    const float sc = (col0 >= scale_begin && col0 < scale_end) ? scale : 1.0f;
     if (bias != nullptr) {
       const uint4* bp = reinterpret_cast<const uint4*>(bias + col0);
 #pragma unroll
@@ -293,14 +296,15 @@ struct LinearEpilogue {
         const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float lo = __uint_as_float(acc[q * 8 + 2 * i]) + bf16_lo(bw[i]);
-          const float hi = __uint_as_float(acc[q * 8 + 2 * i + 1]) + bf16_hi(bw[i]);
+          const float lo = (__uint_as_float(acc[q * 8 + 2 * i]) + bf16_lo(bw[i])) * sc;
+          const float hi = (__uint_as_float(acc[q * 8 + 2 * i + 1]) + bf16_hi(bw[i])) * sc;
           packed[q * 4 + i] = pack_bf16(lo, hi);
         }
       }
     } else {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) packed[i] = pack_bf16(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
+      for (int i = 0; i < 32; ++i)
+        packed[i] = pack_bf16(__uint_as_float(acc[2 * i]) * sc, __uint_as_float(acc[2 * i + 1]) * sc);
     }
   }
 };

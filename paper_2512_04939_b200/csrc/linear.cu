@@ -9,7 +9,14 @@ namespace lv {
 
 cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k, const __nv_bfloat16* w,
                           long long n, const __nv_bfloat16* bias, __nv_bfloat16* out, cudaStream_t s, int* launches) {
+  return launch_linear_scaled(ctx, a, m, k, w, n, bias, 0, 0, 1.0f, out, s, launches);
+}
+
+cudaError_t launch_linear_scaled(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k,
+                                 const __nv_bfloat16* w, long long n, const __nv_bfloat16* bias, int scale_begin,
+                                 int scale_end, float scale, __nv_bfloat16* out, cudaStream_t s, int* launches) {
   if (m == 0) return cudaSuccess;
+  if (scale_begin % 64 != 0 || scale_end % 64 != 0) return cudaErrorInvalidValue;
   CUtensorMap tmap_a, tmap_b, tmap_out;
   if (!make_tmap_bf16_2d(ctx->encode_tiled, &tmap_a, a, (uint64_t)k, (uint64_t)m, (uint64_t)k, kGemmBK, kGemmBM) ||
       !make_tmap_bf16_2d(ctx->encode_tiled, &tmap_b, w, (uint64_t)k, (uint64_t)n, (uint64_t)k, kGemmBK, kGemmBN) ||
@@ -20,6 +27,9 @@ cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m
   epi.bias = bias;
   epi.m_rows = (int)m;
   epi.n_cols = (int)n;
+  epi.scale_begin = scale_begin;
+  epi.scale_end = scale_end;
+  epi.scale = scale;
   static std::atomic<unsigned long long> smem_set{0};
   cudaError_t e = set_max_dynamic_smem_once(reinterpret_cast<const void*>(gemm_tc_kernel<LinearEpilogue>), kGemmSmemBytes,
                                             smem_set);

@@ -126,6 +126,12 @@ qk_embed_kernel(__nv_bfloat16* __restrict__ qkv, const int* __restrict__ kept_id
         v[e] = fmaf(partner, sn[e], v[e] * cs[e]);
       }
     }
+    if (is_k) {
+      // the attention kernel expects K with the softmax scale folded in (the projection before this
+      // pass left it out, so that the normalisation sees K itself)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] *= kKeyScaleLog2e;
+    }
     base[step * 32 + lane] = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
                                         pack_bf16(v[6], v[7]));
   }

@@ -40,6 +40,12 @@ inline cudaError_t set_max_dynamic_smem_once(const void* kernel, int bytes, std:
   return e;
 }
 
+// The attention kernels take the exponentials in base 2 of scores that already carry the softmax
+// scale: 1/sqrt(64) log2(e) is folded into K where K is last rounded to bf16 (the QKV projection's
+// epilogue, or the Q/K normalisation pass), so that no arithmetic stands between the tensor core's
+// scores and the exponential, at no extra rounding.
+constexpr float kKeyScaleLog2e = 0.125f * 1.4426950408889634f;
+
 constexpr long long kMlpChunkRows = 131072;  // rows of the 4D-wide hidden activations held at a time (1 GiB)
 
 // One device allocation carved into named regions.
@@ -186,6 +192,11 @@ cudaError_t launch_unmerge(const litevggt_ctx* ctx, const litevggt_plan* plan, c
 // linear.cu
 cudaError_t launch_linear(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k, const __nv_bfloat16* w,
                           long long n, const __nv_bfloat16* bias, __nv_bfloat16* out, cudaStream_t s, int* launches);
+// The same with output columns [scale_begin, scale_end) (multiples of 64) multiplied by `scale` in
+// fp32 before the one rounding to bf16: the QKV projection of an attention layer scales its K columns.
+cudaError_t launch_linear_scaled(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k,
+                                 const __nv_bfloat16* w, long long n, const __nv_bfloat16* bias, int scale_begin,
+                                 int scale_end, float scale, __nv_bfloat16* out, cudaStream_t s, int* launches);
 
 cudaError_t launch_linear_mlp(litevggt_ctx* ctx, const __nv_bfloat16* a, long long m, long long k,
                               const __nv_bfloat16* w, long long n, const __nv_bfloat16* bias, int gelu,

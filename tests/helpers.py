@@ -27,6 +27,30 @@ LAYER_NOISE = 1e-2
 CORE_NOISE = 4e-3
 
 
+# The library keeps K, wherever it is last rounded to bf16 (QKV projection, Q/K normalisation pass),
+# multiplied by the softmax scale in base-2 units, 1/sqrt(64) * log2(e) in float32, so that its
+# attention kernels can take 2^(q . k) directly.  The oracle knows nothing of this: a K taken from
+# the library's buffers is divided by the constant before it is handed to the oracle, and a K
+# computed by the oracle is multiplied by it before it is compared with the library's.
+K_FOLD = float(np.float32(0.125) * np.float32(1.4426950408889634))
+
+
+def unfold_k(qkv: np.ndarray) -> np.ndarray:
+    """Copy of a [M, 3D] (or one head's [M, 3 dh]) qkv array with the K third divided by K_FOLD."""
+    out = np.array(qkv, dtype=np.float64, copy=True)
+    d = out.shape[1] // 3
+    out[:, d:2 * d] /= K_FOLD
+    return out
+
+
+def fold_k(qkv: np.ndarray) -> np.ndarray:
+    """The opposite direction: an oracle-made qkv with its K third multiplied by K_FOLD."""
+    out = np.array(qkv, dtype=np.float64, copy=True)
+    d = out.shape[1] // 3
+    out[:, d:2 * d] *= K_FOLD
+    return out
+
+
 def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 

@@ -98,10 +98,11 @@ def _check_plan_against_oracle(tag, ctx, plan, x, grad64, wl, interval_layer):
            near_ties_accepted=int((~agree).sum()), margin_below_1e_3=float((margin < 1e-3).mean()),
            margin_below_1e_4=float((margin < 1e-4).mean()), margin_below_1e_5=float((margin < 1e-5).mean()))
     assert np.all(agree[margin > 1e-3]), f"{tag}: argmax differs although the oracle's margin exceeds 1e-3"
-    # 99.9 % agreement; on a population of a few hundred rows (config C1 has 501 src tokens) that is
-    # less than one row, so one near-tie (similarity within 1e-5 of the oracle's best, below) may differ
-    assert (~agree).sum() <= max(1, int(1e-3 * agree.size)), f"{tag}: {(~agree).sum()} of {agree.size} matches differ"
+    # a row that differs must be a near-tie: its similarity within 1e-5 of the oracle's best.  The
+    # 99.9 % clause is applied by the callers to all the plans of a run together: one plan of config
+    # C1 has 501 src rows, of which 99.9 % is less than one row
     assert np.abs(ex["best_sim"] - sim1).max() <= 1e-5, tag
+    ex["match_rows"], ex["match_differences"] = int(agree.size), int((~agree).sum())
     n_remove = O.derived_sizes(wl.frames, wl.grid_h, wl.grid_w, merge_ratio=wl.merge_ratio)["R"]
     dst_of, size, kept = O.select_and_index(ex["cls"], ex["best_dst"], ex["best_sim"], n_remove)
     assert np.array_equal(ex["dst_of"], dst_of) and np.array_equal(ex["size"], size), tag
@@ -133,6 +134,7 @@ def test_plan_refreshed_in_place_on_drifted_features_c4_schedule():
     rows = np.unique(np.concatenate([rng.choice(m, 40, replace=False), [0, m - 1]]))
     toks = np.unique(np.concatenate([rng.choice(ctx.n_tokens, 200, replace=False), [0, ctx.n_tokens - 1]]))
     plan, builds, ex, first = None, 0, None, None
+    rows_seen = differences = 0
     for layer in range(wl.global_layers):
         assert bool(ctx.should_refresh(plan, layer)) == (plan is None or O.should_refresh(layer, 6))
         if ctx.should_refresh(plan, layer):
@@ -142,6 +144,7 @@ def test_plan_refreshed_in_place_on_drifted_features_c4_schedule():
             builds += 1
             ctx.poll()
             ex = _check_plan_against_oracle("C4x32", ctx, plan, x, grad64, wl, layer)
+            rows_seen, differences = rows_seen + ex["match_rows"], differences + ex["match_differences"]
             if first is None:
                 first = ex
             else:
@@ -161,6 +164,7 @@ def test_plan_refreshed_in_place_on_drifted_features_c4_schedule():
         check_bf16(f"C4x32 layer {layer}: unmerge with residual", to_f64(out)[toks], ref_out, sampled=True)
         x = out
     assert builds == 2
+    assert differences <= 1e-3 * rows_seen, f"{differences} of {rows_seen} matches differ from the oracle's"
     plan.destroy()
     ctx.close()
 
@@ -189,6 +193,7 @@ def test_recompute_intervals_of_the_caching_ablation(interval):
     x = tokens.cuda()
     grad = ctx.grad_map(images.cuda())
     plan, builds, ex = None, 0, None
+    rows_seen = differences = 0
     for layer in range(24):
         want = O.should_refresh(layer, interval)
         assert bool(ctx.should_refresh(plan, layer)) == bool(want or plan is None)
@@ -197,6 +202,7 @@ def test_recompute_intervals_of_the_caching_ablation(interval):
             builds += 1
             ctx.poll()
             ex = _check_plan_against_oracle(f"C1 interval {interval}", ctx, plan, x, grad64, wl, layer)
+            rows_seen, differences = rows_seen + ex["match_rows"], differences + ex["match_differences"]
         w = [t.cuda() for t in make_attention_weights(wl, layer)]
         xm = ctx.merge(plan, x)
         ym = ctx.global_attn(xm, *w)
@@ -211,5 +217,7 @@ def test_recompute_intervals_of_the_caching_ablation(interval):
                        O.unmerge(ref_y, ex["dst_of"], x64), noise=LAYER_NOISE / 2)
         x = out
     assert builds == _golden_schedule()[interval]
+    # 99.9 % of all the matches of the run (with a single plan of 501 rows: at most one near-tie)
+    assert differences <= max(1, int(1e-3 * rows_seen)), f"{differences} of {rows_seen} matches differ from the oracle's"
     plan.destroy()
     ctx.close()

@@ -11,7 +11,7 @@ import torch
 import oracle as O
 from synthdata import (WORKLOADS, make_attention_weights, make_block_weights, make_images,
                        make_peaked_attention_inputs, make_tokens)
-from helpers import CORE_NOISE, LAYER_NOISE, bf16_bound, check_bf16, rel_err, report, to_f64
+from helpers import CORE_NOISE, K_FOLD, LAYER_NOISE, bf16_bound, check_bf16, fold_k, rel_err, report, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -172,7 +172,7 @@ def test_attention_layer_on_sampled_rows(run):
     qkv_gpu = ctx.debug_buffer(0)
     o_gpu = ctx.debug_buffer(1)
     # projections on the sampled rows
-    ref_qkv = O.linear(to_f64(xm[rows_t]), w_qkv, b_qkv)
+    ref_qkv = fold_k(O.linear(to_f64(xm[rows_t]), w_qkv, b_qkv))
     check_bf16(f"{run['wl'].name}: qkv projection", to_f64(qkv_gpu[rows_t]), ref_qkv, sampled=True)
     o_rows = to_f64(o_gpu[rows_t])
     ref_y = O.linear(o_rows, w_o, b_o)
@@ -182,7 +182,7 @@ def test_attention_layer_on_sampled_rows(run):
     for head in (0, 6, 15):
         cols = torch.arange(64, device="cuda") + 64 * head
         q = to_f64(qkv_gpu[:, cols])
-        k = to_f64(qkv_gpu[:, 1024 + cols])
+        k = to_f64(qkv_gpu[:, 1024 + cols]) / K_FOLD  # the library's K carries the softmax scale
         v = to_f64(qkv_gpu[:, 2048 + cols])
         ref_o = O.attention_core(np.concatenate([q, k, v], axis=1), heads=1, rows=rows)
         check_bf16(f"{run['wl'].name}: attention core, stock weights, head {head}", o_rows[:, 64 * head:64 * head + 64],
@@ -224,7 +224,7 @@ def test_attention_core_with_peaked_softmax_across_key_chunks(name):
     o_rows = to_f64(o_gpu[rows_t])
     for head in (0, 9, 15):
         cols = torch.arange(64, device="cuda") + 64 * head
-        qkv_h = np.concatenate([to_f64(qkv_gpu[:, cols]), to_f64(qkv_gpu[:, 1024 + cols]),
+        qkv_h = np.concatenate([to_f64(qkv_gpu[:, cols]), to_f64(qkv_gpu[:, 1024 + cols]) / K_FOLD,
                                 to_f64(qkv_gpu[:, 2048 + cols])], axis=1)
         ref_o = O.attention_core(qkv_h, heads=1, rows=rows)
         got = o_rows[:, 64 * head:64 * head + 64]
@@ -297,6 +297,8 @@ def test_qk_norm_and_rope_on_sampled_rows(run):
     for name, c0, g, b in (("Q", 0, affine[0], affine[1]), ("K", 1024, affine[2], affine[3])):
         part = ref[:, c0:c0 + 1024].reshape(len(rows), 16, 64)
         part = O.rope_2d(O.qk_norm(part, to_f64(g), to_f64(b), 1e-5), pos, 100.0).reshape(len(rows), 1024)
+        if name == "K":
+            part = part * K_FOLD
         assert rel_err(got[:, c0:c0 + 1024], part) <= 2 * bf16_bound(part), name
     assert rel_err(got[:, 2048:], ref[:, 2048:]) <= bf16_bound(ref[:, 2048:]), "V is only projected"
     ref_y = O.linear(to_f64(ctx.debug_buffer(1)[rows_t]), to_f64(w_o), to_f64(b_o))
@@ -346,7 +348,7 @@ def test_fp8_attention_variant_on_sampled_rows(name):
     for head in (0, 9, 15):
         sl = slice(64 * head, 64 * head + 64)
         q = decode(f8["q8"][:, sl].cpu().numpy()) * scales[0, head]
-        k = decode(f8["k8"][:, sl].cpu().numpy()) * scales[1, head]
+        k = decode(f8["k8"][:, sl].cpu().numpy()) * scales[1, head] / K_FOLD
         v = decode(f8["v8t"][sl, :m].cpu().numpy().T) * scales[2, head]
         ref_o = O.attention_core(np.concatenate([q, k, v], axis=1), heads=1, rows=rows)
         check_bf16(f"fp8 {name}: attention core, peaked softmax, head {head}", o_rows[:, sl], ref_o, noise=FP8_PEAKED_NOISE,

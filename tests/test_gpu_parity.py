@@ -8,7 +8,8 @@ import torch
 import oracle as O
 from synthdata import (WORKLOADS, Workload, make_attention_weights, make_block_weights, make_images,
                        make_peaked_attention_inputs, make_tokens)
-from helpers import CORE_NOISE, LAYER_NOISE, bf16_bound, bf16_round, check_bf16, rel_err, report, to_f64
+from helpers import (CORE_NOISE, K_FOLD, LAYER_NOISE, bf16_bound, bf16_round, check_bf16, fold_k, rel_err, report,
+                     to_f64, unfold_k)
 
 pytestmark = pytest.mark.gpu
 
@@ -321,12 +322,13 @@ def test_linear(lib, m, k, n):
 
 
 def score_bounds(qkv, heads=16):
-    """Cauchy-Schwarz bound |q| max_k |k| / sqrt(dh) * log2(e) on the base-2 scores of every
-    (row, head): which of the kernel's two softmax forms a row takes depends on it."""
+    """Cauchy-Schwarz bound |q| max_k |k| on the base-2 scores of every (row, head), from the
+    library's own qkv buffer (whose K carries the softmax scale): which of the kernel's two softmax
+    forms a row takes depends on it."""
     m, d = qkv.shape[0], qkv.shape[1] // 3
     q = qkv[:, :d].reshape(m, heads, d // heads)
     k = qkv[:, d:2 * d].reshape(m, heads, d // heads)
-    return np.sqrt((q * q).sum(-1)) * np.sqrt((k * k).sum(-1)).max(0) / np.sqrt(d // heads) * np.log2(np.e)
+    return np.sqrt((q * q).sum(-1)) * np.sqrt((k * k).sum(-1)).max(0)
 
 
 FIXED_REF_LIMIT = 48.0  # the library's kFaFixedRefLimit
@@ -349,7 +351,7 @@ def test_global_attention(lib, wl):
         y = ctx.global_attn(xm.cuda(), wq.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
         ctx.poll()
         # each stage against the oracle fed with the GPU's own upstream (bf16) result
-        ref_qkv = O.linear(to_f64(xm), to_f64(wq), to_f64(b_qkv))
+        ref_qkv = fold_k(O.linear(to_f64(xm), to_f64(wq), to_f64(b_qkv)))
         qkv = to_f64(ctx.debug_buffer(0))
         check_bf16(f"{wl.name}/{tag}: qkv projection", qkv, ref_qkv)
         b = score_bounds(qkv)
@@ -358,7 +360,7 @@ def test_global_attention(lib, wl):
             assert b.max() <= FIXED_REF_LIMIT  # every row takes the fixed-reference form
         else:
             assert (b > FIXED_REF_LIMIT).mean() > 0.5  # most warps take the online form
-        ref_o = O.attention_core(qkv, heads=16)
+        ref_o = O.attention_core(unfold_k(qkv), heads=16)
         o = to_f64(ctx.debug_buffer(1))
         check_bf16(f"{wl.name}/{tag}: attention core", o, ref_o, elem_noise=CORE_NOISE)
         ref_y = O.linear(o, to_f64(w_o), to_f64(b_o))
@@ -386,7 +388,8 @@ def test_attention_core_with_peaked_softmax(lib, grid, sharpness, form):
     report(f"peaked m={m} s={sharpness}: score bound", max=b.max(), min=b.min())
     share_fixed = float((b <= FIXED_REF_LIMIT).mean())
     assert share_fixed > 0.9 if form == "fixed" else share_fixed < 0.5
-    ref_o = O.attention_core(qkv, heads=16)
+    qkv_o = unfold_k(qkv)
+    ref_o = O.attention_core(qkv_o, heads=16)
     o = to_f64(ctx.debug_buffer(1))
     check_bf16(f"peaked m={m} s={sharpness}: attention core", o, ref_o, elem_noise=CORE_NOISE)
     # the case is what it claims to be: the rows of a query's own group hold most of its mass, so
@@ -395,7 +398,7 @@ def test_attention_core_with_peaked_softmax(lib, grid, sharpness, form):
     keep = np.ones(m, bool)
     keep[256:384] = False
     rows = np.flatnonzero(keep)[:200]
-    short = qkv[keep]
+    short = qkv_o[keep]
     ref_short = O.attention_core(short, heads=16, rows=np.arange(200))
     assert rel_err(o[rows], ref_short) > 20 * bf16_bound(ref_o)
     check_bf16(f"peaked m={m} s={sharpness}: output projection", to_f64(y), O.linear(o, to_f64(w_o), to_f64(b_o)))
@@ -434,6 +437,7 @@ def test_global_attention_with_qk_norm_and_rope(lib, wl, mode):
     # the transformed Q and K against the oracle's (two roundings on the GPU side: the projection's
     # output and the transformed values; V must be untouched)
     ref_y, ref_qkv, _ = O.global_attention(xm64, *w64, heads=16, return_parts=True, ext=ext)
+    ref_qkv = fold_k(ref_qkv)
     qkv = to_f64(ctx.debug_buffer(0))
     d = 1024
     for name, sl in (("Q", slice(0, d)), ("K", slice(d, 2 * d)), ("V", slice(2 * d, 3 * d))):
@@ -442,10 +446,10 @@ def test_global_attention_with_qk_norm_and_rope(lib, wl, mode):
         # RMS after rotating pairs in which a small entry inherits the rounding of a large partner
         second = 0.0 if name == "V" else 1.25 * rel_err(bf16_round(ref_qkv[:, sl]), ref_qkv[:, sl])
         check_bf16(f"{wl.name}/{mode}: {name}", qkv[:, sl], ref_qkv[:, sl], noise=second)
-    plain = to_f64(ctx.linear(xm, w_qkv.cuda(), b_qkv.cuda()))
+    plain = fold_k(to_f64(ctx.linear(xm, w_qkv.cuda(), b_qkv.cuda())))
     assert np.array_equal(qkv[:, 2 * d:], plain[:, 2 * d:])
     # the core on the GPU's own transformed Q/K/V, and the layer end to end
-    ref_o = O.attention_core(qkv, heads=16)
+    ref_o = O.attention_core(unfold_k(qkv), heads=16)
     check_bf16(f"{wl.name}/{mode}: attention core", to_f64(ctx.debug_buffer(1)), ref_o, elem_noise=CORE_NOISE)
     # one more stored rounding than the plain layer (the transformed Q and K)
     check_bf16(f"{wl.name}/{mode}: layer end to end", to_f64(y), ref_y, noise=LAYER_NOISE)
@@ -725,11 +729,11 @@ def test_fp8_attention_variant(lib, wl):
         assert np.array_equal(got_codes[nonzero], codes_ref[nonzero]) and np.all((got_codes[~nonzero] & 0x7f) == 0)
         assert np.all(f8["v8t"].cpu().numpy()[:, m:] == 0), "padded keys must be zero"
         # the core on the dequantised operands
-        ref_o = O.attention_core(deq_ref, heads=16)
+        ref_o = O.attention_core(unfold_k(deq_ref), heads=16)
         o = to_f64(ctx.debug_buffer(1))
         check_bf16(f"fp8 {wl.name}/{tag}: attention core", o, ref_o, noise=noise)
         # against the unquantised core: what the 8-bit operands cost (reported, loosely bounded)
-        ref_o_bf16 = O.attention_core(qkv, heads=16)
+        ref_o_bf16 = O.attention_core(unfold_k(qkv), heads=16)
         report(f"fp8 {wl.name}/{tag}: attention core vs unquantised operands", err_over_rms=rel_err(o, ref_o_bf16))
         assert rel_err(o, ref_o_bf16) < (0.1 if tag == "stock" else 1.0)
         check_bf16(f"fp8 {wl.name}/{tag}: output projection", to_f64(y), O.linear(o, to_f64(w_o), to_f64(b_o)))
@@ -745,6 +749,7 @@ def test_fp8_attention_variant_with_peaked_softmax(lib):
     ctx.global_attn(x.cuda(), w_qkv.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
     ctx.poll()
     deq, _, _ = O.quantize_qkv_e4m3(to_f64(ctx.debug_buffer(0)), heads=16)
+    deq = unfold_k(deq)
     ref_o = O.attention_core(deq, heads=16)
     o = to_f64(ctx.debug_buffer(1))
     check_bf16("fp8 peaked: attention core", o, ref_o, noise=FP8_PEAKED_NOISE)
