@@ -292,7 +292,6 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   const size_t o_keys = c.take<unsigned long long>(cap);
   const size_t o_tmp = c.take<int>(z.n_tokens + 1), o_blk = c.take<int>(2048), o_row = c.take<int>(z.n_tokens);
   const size_t o_qkv = c.take<__nv_bfloat16>(z.n_merged * 3 * z.dim), o_o = c.take<__nv_bfloat16>(z.n_merged * z.dim);
-  const size_t o_vparts = c.take<float>(4 * fp);
   size_t ml_off = 0;
   const size_t state_bytes = attention_state_bytes(z.n_merged, z.dim, z.heads, &ml_off);
   const size_t o_state = c.take<uint8_t>((long long)state_bytes);
@@ -324,7 +323,6 @@ litevggt_status litevggt_create(const litevggt_config* cfg, int device, litevggt
   ws.row_of = reinterpret_cast<int*>(ws.base + o_row);
   ws.qkv = reinterpret_cast<__nv_bfloat16*>(ws.base + o_qkv);
   ws.attn_o = reinterpret_cast<__nv_bfloat16*>(ws.base + o_o);
-  ws.var_parts = reinterpret_cast<float*>(ws.base + o_vparts);
   if (state_bytes > 0) {
     ws.attn_o_state = reinterpret_cast<float*>(ws.base + o_state);
     ws.attn_ml_state = reinterpret_cast<float*>(ws.base + o_state + ml_off);
@@ -473,7 +471,7 @@ litevggt_status litevggt_merge_plan(litevggt_ctx* ctx, const void* x, const floa
   cudaError_t e;
   {
     StepTimer t(ctx, 1, s);
-    e = launch_var_map(ctx, xb, ctx->ws.var_parts, ctx->ws.var_map, s, &n);
+    e = launch_var_map(ctx, xb, ctx->ws.var_map, s, &n);
   }
   if (e == cudaSuccess) {
     StepTimer t(ctx, 2, s);

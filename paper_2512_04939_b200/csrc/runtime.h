@@ -54,7 +54,6 @@ struct Workspace {
   size_t bytes = 0;
   // scoring
   float* var_map = nullptr;     // [F*P]
-  float* var_parts = nullptr;   // [4][F*P] per-channel-quarter partial sums of the Var map
   float* ga_score = nullptr;    // [F*P]
   uint8_t* cls = nullptr;       // [N]
   int* src_list = nullptr;      // [|Src|] token index, ascending
@@ -168,7 +167,7 @@ bool make_tmap_u8_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64
 
 // scoring.cu
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches);
-cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var_parts, float* var,
+cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var,
                            cudaStream_t s, int* launches);
 cudaError_t launch_partition(const litevggt_ctx* ctx, const float* grad, const float* var, float* ga, uint8_t* cls,
                              cudaStream_t s, int* launches);

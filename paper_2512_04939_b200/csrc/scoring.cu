@@ -123,216 +123,198 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 // anything is squared).  So only the per-channel box sums of d are needed, plus a box sum of the
 // scalar |d_j|^2 - not a second per-channel box filter.
 //
-// A warp owns 16 channels of a block of 30 grid rows (+ one halo row on either side) and walks along
-// the rows, one grid column per step.  The column's 32 tokens (32 bytes each) arrive in the warp's own
-// ring in shared memory by asynchronous copies, two lanes per token, kVarDepth columns ahead; rows
-// outside the grid are filled with x0, so they contribute d = 0 and the clipped window needs no
-// special case.  Lane = grid row: it reads its own token and the ones above and below from the ring
-// (48-byte row pitch: conflict-free 16-byte reads), forms the vertical sums of d and of |d|^2, and
-// keeps the last three columns in registers, from which the window sums of the column before follow.
-// Scattered 16-byte global loads and two shuffles per channel cost this kernel's first version
-// (lane loads its own token, neighbours by shuffle) three times the L1 wavefronts.  No barrier
-// inside the walk; only __syncwarp around the ring.  A warp makes four such passes (64 channels),
-// adding its results up in its own shared-memory rows; the four warps of a CTA cover a quarter of
-// the channels and are added in a fixed order into that quarter's plane, and var_sum_kernel adds the
-// four planes, so the map is deterministic.
+// The step costs about nine fp32 operations per channel of a token (difference, square, two adds
+// down the rows, two along them, square of the window sum, with the halo rows on top), which at the
+// rate of the FMA pipes is as long as reading the token from HBM: the kernel has to be lean in
+// instructions, not only in bytes.  A CTA owns a strip of kVarRows grid rows of one frame, its four
+// warps a quarter of the channels each; lane = 8 consecutive channels, so a token's quarter is one
+// fully coalesced 512-byte load straight into registers, with no shared-memory stage and no
+// barrier.  The warp walks along the strip one grid column per step: the column's kVarRows + 2
+// tokens (one halo row above and below; outside the grid the lane's own x0 stands in, so d = 0)
+// are converted once, give the column's vertical sums of d and of |d|^2, and the sums of the two
+// columns before stay in registers; the loads of the next column are issued as soon as this
+// column's registers are free.  A window's value, (1/n) sum |d|^2 - (1/n^2) |sum d|^2, is linear in
+// the per-lane partial sums over the channels, so each lane forms it for its 8 channels, a
+// butterfly over the warp adds the 32 lanes for all rows of the strip at once, the four warps'
+// sums meet in shared memory and are added in a fixed order: the map is deterministic.
 #ifndef LV_VAR_OCC
-#define LV_VAR_OCC 4
-#endif
-#ifndef LV_VAR_DEPTH
-#define LV_VAR_DEPTH 4
+#define LV_VAR_OCC 3
 #endif
 constexpr int kVarThreads = 128;
 constexpr int kVarWarps = kVarThreads / 32;
-constexpr int kVarChannels = 256;     // per CTA
-constexpr int kVarPassChannels = 16;  // per warp pass
-constexpr int kVarRowsPerBlock = 30;
+constexpr int kVarRows = 4;  // grid rows per CTA
 constexpr int kVarMaxW = 64;
-constexpr int kVarDepth = LV_VAR_DEPTH;  // grid columns in flight
-constexpr int kVarRowPitch = 48;         // bytes per token in the ring: 32 of data + 16 against bank conflicts
-constexpr int kVarSlotBytes = 32 * kVarRowPitch;
-// dynamic shared memory per warp: the ring [depth][32 rows][48 B], then this warp's results
-// [32 lanes][grid_w + 1]
-__host__ __device__ inline size_t var_warp_smem_bytes(int grid_w) {
-  return (size_t)kVarDepth * kVarSlotBytes + (size_t)32 * (grid_w + 1) * sizeof(float);
-}
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int kPending>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
-}
+constexpr int kVarTokenVec = 128;  // 16-byte vectors per token
 
 struct VarColumn {
-  float2 s[kVarPassChannels / 2];  // vertical 3-sum of d, per channel (pairs: packed fp32 arithmetic)
-  float q;                         // vertical 3-sum of |d|^2
+  float2 s[kVarRows][4];  // vertical 3-sums of d, this lane's 8 channels as pairs (packed fp32 arithmetic)
+  float q[kVarRows];      // vertical 3-sums of this lane's share of |d|^2
 };
 
-__global__ void __launch_bounds__(kVarThreads, LV_VAR_OCC)
-var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var_parts, int frames, int grid_h, int grid_w,
-               int n_special) {
-  extern __shared__ __align__(16) uint8_t var_smem[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const size_t warp_bytes = var_warp_smem_bytes(grid_w);
-  uint8_t* ring = var_smem + warp * warp_bytes;
-  const int acc_pitch = grid_w + 1;
-  float* acc = reinterpret_cast<float*>(ring + kVarDepth * kVarSlotBytes) + lane * acc_pitch;  // this lane's results
-  const int quarter = blockIdx.x, f = blockIdx.z;
-  const int row0 = blockIdx.y * kVarRowsPerBlock - 1;  // grid row of lane 0 (a halo row)
-  const int row = row0 + lane;
-  const bool row_valid = row >= 0 && row < grid_h;
-  const bool emits = row_valid && lane >= 1 && lane <= kVarRowsPerBlock;
-  const int tokens_frame = grid_h * grid_w + n_special;
-  const __nv_bfloat16* frame = x + ((size_t)f * tokens_frame + n_special) * 1024;
-  const float inv_rows = 1.0f / (float)(1 + (row > 0 ? 1 : 0) + (row < grid_h - 1 ? 1 : 0));
-  // as a copier, this lane moves 16 bytes of two tokens per column: rows row0 + lane/2 and + 16
-  const int half = lane & 1;
-  const int crow_a = row0 + (lane >> 1), crow_b = crow_a + 16;
-  const bool cvalid_a = crow_a >= 0 && crow_a < grid_h, cvalid_b = crow_b >= 0 && crow_b < grid_h;
-  // lanes 0 and 31 have no row above / below in the ring: they read their own row instead; what they
-  // compute is never emitted
-  const int up = lane > 0 ? lane - 1 : lane, dn = lane < 31 ? lane + 1 : lane;
+__device__ __forceinline__ void var_zero(VarColumn& c) {
+#pragma unroll
+  for (int r = 0; r < kVarRows; ++r) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c.s[r][i] = make_float2(0.0f, 0.0f);
+    c.q[r] = 0.0f;
+  }
+}
 
-  for (int pass = 0; pass < kVarChannels / kVarWarps / kVarPassChannels; ++pass) {
-    // In one pass the four warps take the four 32-byte sectors of the same 128-byte lines, so a line
-    // comes from HBM once and the other three warps find it in cache.
-    const int ch = quarter * kVarChannels + (pass * kVarWarps + warp) * kVarPassChannels;
-    const __nv_bfloat16* x0_ptr = frame + ch;  // first patch token of the frame, this pass's channels
-    float2 x0[kVarPassChannels / 2], x0_3[kVarPassChannels / 2];
-    {
-      const uint4* p0 = reinterpret_cast<const uint4*>(x0_ptr);
-      const uint4 a = __ldg(p0), b = __ldg(p0 + 1);
-      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+// Vertical sums of the column held in raw[] (kVarRows + 2 tokens, top halo first) into `out`.
+__device__ __forceinline__ void var_column(const uint4 (&raw)[kVarRows + 2], const float2 (&neg_x0)[4], VarColumn& out) {
+  float2 d[kVarRows + 2][4];
+  float q[kVarRows + 2];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        x0[i] = make_float2(bf16_lo(w[i]), bf16_hi(w[i]));
-        x0_3[i] = make_float2(-3.0f * x0[i].x, -3.0f * x0[i].y);
-      }
+  for (int r = 0; r < kVarRows + 2; ++r) {
+    const uint32_t w[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
+    float2 q2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      d[r][i] = __fadd2_rn(make_float2(bf16_lo(w[i]), bf16_hi(w[i])), neg_x0[i]);
+      q2 = __ffma2_rn(d[r][i], d[r][i], q2);
     }
-    const __nv_bfloat16* src_a = cvalid_a ? frame + (size_t)crow_a * grid_w * 1024 + ch + half * 8 : nullptr;
-    const __nv_bfloat16* src_b = cvalid_b ? frame + (size_t)crow_b * grid_w * 1024 + ch + half * 8 : nullptr;
-    // column px into its slot of the ring; one copy group per column (empty past the last column), so
-    // the number of groups still pending tells which columns have landed
-    auto fetch = [&](int px) {
-      if (px < grid_w) {
-        uint8_t* slot = ring + (px % kVarDepth) * kVarSlotBytes + half * 16;
-        cp_async16(slot + (lane >> 1) * kVarRowPitch, src_a != nullptr ? src_a + (size_t)px * 1024 : x0_ptr + half * 8);
-        cp_async16(slot + ((lane >> 1) + 16) * kVarRowPitch,
-                   src_b != nullptr ? src_b + (size_t)px * 1024 : x0_ptr + half * 8);
-      }
-      cp_async_commit();
-    };
+    q[r] = q2.x + q2.y;
+  }
+  // rows r and r + 1 of the strip share the sum of the two tokens between them
 #pragma unroll
-    for (int k = 0; k < kVarDepth; ++k) fetch(k);
-    // the 16 channels of one token of the slot, as 8 pairs
-    auto load_x = [&](const uint8_t* slot, int r, float2 (&v)[kVarPassChannels / 2]) {
-      const uint4* p = reinterpret_cast<const uint4*>(slot + r * kVarRowPitch);
-      const uint4 a = p[0], b = p[1];
-      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+  for (int r = 0; r < kVarRows; r += 2) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = make_float2(bf16_lo(w[i]), bf16_hi(w[i]));
-    };
-    // one grid column: vertical sums over this lane's row and the rows above and below, then the
-    // slot goes back to the copiers.  Rows outside the grid hold x0, so the sum of d over the three
-    // rows is always (sum of x) - 3 x0.
-    auto take = [&](int c, VarColumn& out) {
-      if (c < grid_w) {
-        cp_async_wait<kVarDepth - 1>();  // all but the newest kVarDepth - 1 groups: column c has landed
-        __syncwarp();                     // ... for every lane's copies
-        const uint8_t* slot = ring + (c % kVarDepth) * kVarSlotBytes;
-        float2 v[kVarPassChannels / 2];
-        load_x(slot, lane, v);
-        float2 q2 = make_float2(0.0f, 0.0f);
+    for (int i = 0; i < 4; ++i) {
+      const float2 mid = __fadd2_rn(d[r + 1][i], d[r + 2][i]);
+      out.s[r][i] = __fadd2_rn(mid, d[r][i]);
+      out.s[r + 1][i] = __fadd2_rn(mid, d[r + 3][i]);
+    }
+    const float qm = q[r + 1] + q[r + 2];
+    out.q[r] = qm + q[r];
+    out.q[r + 1] = qm + q[r + 3];
+  }
+}
+
+// The 32 lanes' values of all four rows added up: afterwards every lane holds the sum for row lane >> 3.
+__device__ __forceinline__ float var_reduce_rows(const float (&v)[kVarRows], int lane) {
+  static_assert(kVarRows == 4, "the butterfly below is written for four rows");
+  const bool hi = (lane & 16) != 0;
+  const float a0 = (hi ? v[2] : v[0]) + __shfl_xor_sync(0xffffffffu, hi ? v[0] : v[2], 16);
+  const float a1 = (hi ? v[3] : v[1]) + __shfl_xor_sync(0xffffffffu, hi ? v[1] : v[3], 16);
+  const bool hi2 = (lane & 8) != 0;
+  float b = (hi2 ? a1 : a0) + __shfl_xor_sync(0xffffffffu, hi2 ? a0 : a1, 8);
+  b += __shfl_xor_sync(0xffffffffu, b, 4);
+  b += __shfl_xor_sync(0xffffffffu, b, 2);
+  b += __shfl_xor_sync(0xffffffffu, b, 1);
+  return b;
+}
+
+__global__ void __launch_bounds__(kVarThreads, LV_VAR_OCC)
+var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var, int grid_h, int grid_w, int n_special) {
+  __shared__ float part[kVarWarps][kVarRows][kVarMaxW];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int f = blockIdx.y, row_base = blockIdx.x * kVarRows;
+  const int tokens_frame = grid_h * grid_w + n_special;
+  // this lane's 8 channels of the frame's first patch token
+  const uint4* frame = reinterpret_cast<const uint4*>(x + ((size_t)f * tokens_frame + n_special) * 1024) + warp * 32 + lane;
+  const uint4 x0_raw = __ldg(frame);
+  float2 neg_x0[4];
+  {
+    const uint32_t w[4] = {x0_raw.x, x0_raw.y, x0_raw.z, x0_raw.w};
 #pragma unroll
-        for (int i = 0; i < kVarPassChannels / 2; ++i) {
-          const float2 d = __fadd2_rn(v[i], make_float2(-x0[i].x, -x0[i].y));
-          q2 = __ffma2_rn(d, d, q2);
-          out.s[i] = __fadd2_rn(v[i], x0_3[i]);
-        }
-        load_x(slot, up, v);
+    for (int i = 0; i < 4; ++i) neg_x0[i] = make_float2(-bf16_lo(w[i]), -bf16_hi(w[i]));
+  }
+  // rows of the column: r = 0 is the halo row above the strip
+  bool row_ok[kVarRows + 2];
+  float inv_rows[kVarRows];
 #pragma unroll
-        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = __fadd2_rn(out.s[i], v[i]);
-        load_x(slot, dn, v);
+  for (int r = 0; r < kVarRows + 2; ++r) {
+    const int row = row_base - 1 + r;
+    row_ok[r] = row >= 0 && row < grid_h;
+  }
 #pragma unroll
-        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = __fadd2_rn(out.s[i], v[i]);
-        const float q = q2.x + q2.y;
-        const float q_up = __shfl_up_sync(0xffffffffu, q, 1), q_dn = __shfl_down_sync(0xffffffffu, q, 1);
-        out.q = q + (lane > 0 ? q_up : 0.0f) + (lane < 31 ? q_dn : 0.0f);
-        __syncwarp();  // every lane has read the slot
-      } else {
+  for (int r = 0; r < kVarRows; ++r)
+    inv_rows[r] = 1.0f / (float)(1 + (row_ok[r] ? 1 : 0) + (row_ok[r + 2] ? 1 : 0));
+  const int row_stride = grid_w * kVarTokenVec;
+  const uint4* col_ptr = frame + (ptrdiff_t)(row_base - 1) * row_stride;  // only dereferenced where row_ok
+
+  uint4 raw[kVarRows + 2];
 #pragma unroll
-        for (int i = 0; i < kVarPassChannels / 2; ++i) out.s[i] = make_float2(0.0f, 0.0f);
-        out.q = 0.0f;
-      }
-      fetch(c + kVarDepth);
-    };
-    // window of grid column px = columns l, m, r (absent ones are all-zero)
-    auto emit = [&](int px, const VarColumn& l, const VarColumn& m, const VarColumn& r) {
+  for (int r = 0; r < kVarRows + 2; ++r) raw[r] = row_ok[r] ? __ldg(col_ptr + (ptrdiff_t)r * row_stride) : x0_raw;
+  // rows outside the grid keep x0 in their registers for the whole walk
+  auto load_next = [&](int c) {
+    if (c < grid_w) {
+      col_ptr += kVarTokenVec;
+#pragma unroll
+      for (int r = 0; r < kVarRows + 2; ++r)
+        if (row_ok[r]) raw[r] = __ldg(col_ptr + (ptrdiff_t)r * row_stride);
+    }
+  };
+  // window of grid column px = columns a, b, c (an absent one is all-zero); `ab` = a + b
+  auto emit = [&](int px, const VarColumn& ab, const VarColumn& c) {
+    const float inv_cols = (px > 0 && px < grid_w - 1) ? (1.0f / 3.0f) : (grid_w > 1 ? 0.5f : 1.0f);
+    float v[kVarRows];
+#pragma unroll
+    for (int r = 0; r < kVarRows; ++r) {
       float2 m2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int i = 0; i < kVarPassChannels / 2; ++i) {
-        const float2 t = __fadd2_rn(__fadd2_rn(l.s[i], m.s[i]), r.s[i]);
+      for (int i = 0; i < 4; ++i) {
+        const float2 t = __fadd2_rn(ab.s[r][i], c.s[r][i]);
         m2 = __ffma2_rn(t, t, m2);
       }
-      const float inv_n = inv_rows * ((px > 0 && px < grid_w - 1) ? (1.0f / 3.0f) : (grid_w > 1 ? 0.5f : 1.0f));
-      const float v = (l.q + m.q + r.q) * inv_n - (m2.x + m2.y) * inv_n * inv_n;
-      if (emits) acc[px] = pass == 0 ? v : acc[px] + v;
-    };
-    VarColumn ca, cb, cc;
-#pragma unroll
-    for (int i = 0; i < kVarPassChannels / 2; ++i) ca.s[i] = make_float2(0.0f, 0.0f);
-    ca.q = 0.0f;
-    take(0, cb);
-    // three columns per trip, so the column sums rotate through fixed registers
-    for (int px = 0; px < grid_w; px += 3) {
-      take(px + 1, cc);
-      emit(px, ca, cb, cc);
-      if (px + 1 < grid_w) {
-        take(px + 2, ca);
-        emit(px + 1, cb, cc, ca);
-      }
-      if (px + 2 < grid_w) {
-        take(px + 3, cb);
-        emit(px + 2, cc, ca, cb);
-      }
+      const float inv_n = inv_rows[r] * inv_cols;
+      v[r] = inv_n * ((ab.q[r] + c.q[r]) - inv_n * (m2.x + m2.y));
     }
-    cp_async_wait<0>();
-    __syncwarp();
+    const float total = var_reduce_rows(v, lane);
+    if ((lane & 7) == 0) part[warp][lane >> 3][px] = total;
+  };
+  // One step: `older` + `newer` are the columns cn - 2 and cn - 1; the column cn, in raw[], replaces
+  // the older one, and the window of column cn - 1 is complete.
+  auto step = [&](VarColumn& older, const VarColumn& newer, int cn) {
+    VarColumn ab;
+#pragma unroll
+    for (int r = 0; r < kVarRows; ++r) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ab.s[r][i] = __fadd2_rn(older.s[r][i], newer.s[r][i]);
+      ab.q[r] = older.q[r] + newer.q[r];
+    }
+    var_column(raw, neg_x0, older);
+    load_next(cn + 1);
+    emit(cn - 1, ab, older);
+  };
+
+  VarColumn ca, cb;
+  var_zero(ca);
+  var_column(raw, neg_x0, cb);  // column 0
+  load_next(1);
+  for (int cn = 1; cn < grid_w; cn += 2) {
+    step(ca, cb, cn);
+    if (cn + 1 < grid_w) step(cb, ca, cn + 1);
+  }
+  {
+    // last column: nothing to its right
+    VarColumn zero;
+    var_zero(zero);
+    VarColumn ab;
+#pragma unroll
+    for (int r = 0; r < kVarRows; ++r) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ab.s[r][i] = __fadd2_rn(ca.s[r][i], cb.s[r][i]);
+      ab.q[r] = ca.q[r] + cb.q[r];
+    }
+    emit(grid_w - 1, ab, zero);
   }
   __syncthreads();
-  // rows of this block, all columns: the four warps' partial sums in a fixed order
-  const int r0 = blockIdx.y * kVarRowsPerBlock;
-  const int n_rows = min(kVarRowsPerBlock, grid_h - r0);
-  float* out = var_parts + ((size_t)quarter * frames + f) * grid_h * grid_w + (size_t)r0 * grid_w;
-  auto warp_acc = [&](int w, int lane_row, int px) {
-    return reinterpret_cast<const float*>(var_smem + w * warp_bytes + kVarDepth * kVarSlotBytes)[lane_row * acc_pitch + px];
-  };
+  // the four channel quarters in a fixed order; mean over the 1024 channels
+  const int n_rows = min(kVarRows, grid_h - row_base);
+  float* out = var + ((size_t)f * grid_h + row_base) * grid_w;
   for (int i = threadIdx.x; i < n_rows * grid_w; i += kVarThreads) {
     const int r = i / grid_w, px = i - r * grid_w;
-    out[i] = ((warp_acc(0, r + 1, px) + warp_acc(1, r + 1, px)) + warp_acc(2, r + 1, px)) + warp_acc(3, r + 1, px);
+    out[i] = (((part[0][r][px] + part[1][r][px]) + part[2][r][px]) + part[3][r][px]) / 1024.0f;
   }
 }
 
-__global__ void var_sum_kernel(const float* __restrict__ parts, float* __restrict__ var, long long count) {
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < count) var[i] = (((parts[i] + parts[count + i]) + parts[2 * count + i]) + parts[3 * count + i]) / 1024.0f;
-}
-
-cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var_parts, float* var,
-                           cudaStream_t s, int* launches) {
+cudaError_t launch_var_map(const litevggt_ctx* ctx, const __nv_bfloat16* x, float* var, cudaStream_t s,
+                           int* launches) {
   const Sizes& z = ctx->sz;
-  const unsigned row_blocks = (unsigned)((z.grid_h + kVarRowsPerBlock - 1) / kVarRowsPerBlock);
-  const int smem = (int)(kVarWarps * var_warp_smem_bytes(z.grid_w));
-  cudaError_t e = cudaFuncSetAttribute(var_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
-  var_map_kernel<<<dim3(4, row_blocks, z.frames), kVarThreads, smem, s>>>(x, var_parts, z.frames, z.grid_h, z.grid_w,
-                                                                         z.n_special);
-  ++*launches;
-  const long long count = (long long)z.frames * z.patches;
-  var_sum_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(var_parts, var, count);
+  if (z.grid_w > kVarMaxW) return cudaErrorInvalidValue;
+  const unsigned strips = (unsigned)((z.grid_h + kVarRows - 1) / kVarRows);
+  var_map_kernel<<<dim3(strips, z.frames), kVarThreads, 0, s>>>(x, var, z.grid_h, z.grid_w, z.n_special);
   ++*launches;
   return cudaGetLastError();
 }
