@@ -15,14 +15,18 @@ namespace lv {
 // shuffle, the separable Sobel pair (per row the horizontal difference r - l and the horizontal
 // smoothing l + 2c + r, kept for the last three rows), the magnitude, a running sum per column.  At
 // the bottom of a patch row the columns of a patch are added by a shuffle tree and one lane writes
-// the patch mean.  Rows are loaded three steps ahead (deeper measured slower); there is no shared
-// memory and no barrier.
+// the patch mean.  Rows are loaded a few steps ahead; there is no shared memory and no barrier.
+// grad_map_kernel takes any patch size up to 30; grad_map_patch_kernel is the same walk for the
+// 14-pixel patches of the model, with a patch's rows unrolled and seven rows in flight.
 constexpr int kGradThreads = 128;
 #ifndef LV_GRAD_PATCH_ROWS
 #define LV_GRAD_PATCH_ROWS 7
 #endif
 #ifndef LV_GRAD_AHEAD
 #define LV_GRAD_AHEAD 3
+#endif
+#ifndef LV_GRAD_AHEAD14
+#define LV_GRAD_AHEAD14 7
 #endif
 constexpr int kGradPatchRows = LV_GRAD_PATCH_ROWS;  // patch rows per warp
 constexpr int kGradAhead = LV_GRAD_AHEAD;           // image rows in flight
@@ -104,6 +108,82 @@ grad_map_kernel(const float* __restrict__ images, float* __restrict__ grad, int 
   }
 }
 
+// The same walk with the patch size known at compile time: the rows of a patch are unrolled, so the
+// row in hand, its place in the load queue and the bottom of the patch are all static and the
+// per-row bookkeeping (row counters, queue index, end-of-patch test) is gone.  kAhead divides kPatch.
+template <int kPatch, int kAhead>
+__global__ void __launch_bounds__(kGradThreads)
+grad_map_patch_kernel(const float* __restrict__ images, float* __restrict__ grad, int grid_h, int grid_w) {
+  static_assert(kPatch % kAhead == 0 && kPatch <= 30 && kAhead >= 2, "queue slots must be static");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int pps = 30 / kPatch;
+  const int strips = (grid_w + pps - 1) / pps;
+  const int strip = blockIdx.x * (kGradThreads / 32) + warp;
+  if (strip >= strips) return;  // whole warp; nothing below synchronises across warps
+  const int f = blockIdx.z;
+  const int pr0 = blockIdx.y * kGradPatchRows;
+  const int pr1 = min(grid_h, pr0 + kGradPatchRows);
+  const int h = grid_h * kPatch, w = grid_w * kPatch;
+  const size_t plane = (size_t)h * w;
+  int x = strip * pps * kPatch - 1 + lane;
+  x = x < 0 ? 0 : (x >= w ? w - 1 : x);
+  const float* col = images + (size_t)f * 3 * plane + x;
+  const bool own = lane >= 1 && lane <= pps * kPatch;
+  const int seg = own ? (lane - 1) / kPatch : 0;
+  const int in_seg = own ? (lane - 1) - seg * kPatch : kPatch;
+  const int patch_x = strip * pps + seg;
+  const bool writer = own && in_seg == 0 && patch_x < grid_w;
+  constexpr float inv_area = 1.0f / (float)(kPatch * kPatch);
+
+  const int y_first = pr0 * kPatch - 1;  // halo row above (clamped when it is outside)
+  float q[kAhead][3];
+  // row i of the walk (0 = halo row above the block); rows past the image repeat its last row
+  auto load_row = [&](int i, float (&dst)[3]) {
+    const int y = min(max(y_first + i, 0), h - 1);
+    const float* p = col + (size_t)y * w;
+    dst[0] = __ldg(p);
+    dst[1] = __ldg(p + plane);
+    dst[2] = __ldg(p + 2 * plane);
+  };
+  struct RowTerms { float d, s; };
+  auto terms = [&](const float (&rgb)[3]) {
+    const float g = (rgb[0] + rgb[1] + rgb[2]) * (1.0f / 3.0f);
+    const float l = __shfl_up_sync(0xffffffffu, g, 1), r = __shfl_down_sync(0xffffffffu, g, 1);
+    return RowTerms{r - l, fmaf(2.0f, g, l + r)};
+  };
+  // rows 0 and 1 come through registers of their own; the queue then holds rows 2 .. kAhead + 1,
+  // so row 2 + k of a patch row sits in slot k % kAhead
+  float first[2][3];
+  load_row(0, first[0]);
+  load_row(1, first[1]);
+#pragma unroll
+  for (int k = 0; k < kAhead; ++k) load_row(2 + k, q[k]);
+  RowTerms t0 = terms(first[0]), t1 = terms(first[1]);
+  int i = 2;  // next row of the walk
+  for (int pr = pr0; pr < pr1; ++pr) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int k = 0; k < kPatch; ++k) {
+      const RowTerms t2 = terms(q[k % kAhead]);
+      load_row(i + k + kAhead, q[k % kAhead]);
+      const float gx = fmaf(2.0f, t1.d, t0.d + t2.d);
+      const float gy = t2.s - t0.s;
+      acc += sqrt_approx(fmaf(gx, gx, gy * gy));
+      t0 = t1;
+      t1 = t2;
+    }
+    i += kPatch;
+    // bottom of a patch row: add the columns of each patch, lowest lane of the patch writes
+    float v = own ? acc : 0.0f;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float t = __shfl_down_sync(0xffffffffu, v, off);
+      if (in_seg + off < kPatch) v += t;
+    }
+    if (writer) grad[((size_t)f * grid_h + pr) * grid_w + patch_x] = v * inv_area;
+  }
+}
+
 cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float* grad, cudaStream_t s, int* launches) {
   const Sizes& z = ctx->sz;
   const int patch = ctx->cfg.patch_px;
@@ -111,7 +191,10 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
   const int strips = (z.grid_w + pps - 1) / pps;
   const dim3 grid((unsigned)((strips + kGradThreads / 32 - 1) / (kGradThreads / 32)),
                   (unsigned)((z.grid_h + kGradPatchRows - 1) / kGradPatchRows), (unsigned)z.frames);
-  grad_map_kernel<<<grid, kGradThreads, 0, s>>>(images, grad, z.grid_h, z.grid_w, patch);
+  if (patch == 14)
+    grad_map_patch_kernel<14, LV_GRAD_AHEAD14><<<grid, kGradThreads, 0, s>>>(images, grad, z.grid_h, z.grid_w);
+  else
+    grad_map_kernel<<<grid, kGradThreads, 0, s>>>(images, grad, z.grid_h, z.grid_w, patch);
   ++*launches;
   return cudaGetLastError();
 }
@@ -131,7 +214,8 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 // fully coalesced 512-byte load straight into registers, with no shared-memory stage and no
 // barrier.  The warp walks along the strip one grid column per step: the column's kVarRows + 2
 // tokens (one halo row above and below; outside the grid the lane's own x0 stands in, so d = 0)
-// are converted once, give the column's vertical sums of d and of |d|^2, and the sums of the two
+// are read once (the difference to x0 comes from a mixed-precision add that takes the bf16 value as
+// it is, so no separate conversion), give the column's vertical sums of d and of |d|^2, and the sums of the two
 // columns before stay in registers; the loads of the next column are issued as soon as this
 // column's registers are free.  A window's value, (1/n) sum |d|^2 - (1/n^2) |sum d|^2, is linear in
 // the per-lane partial sums over the channels, so each lane forms it for its 8 channels, a
@@ -145,6 +229,22 @@ constexpr int kVarWarps = kVarThreads / 32;
 constexpr int kVarRows = 4;  // grid rows per CTA
 constexpr int kVarMaxW = 64;
 constexpr int kVarTokenVec = 128;  // 16-byte vectors per token
+#ifndef LV_VAR_PREFETCH
+#define LV_VAR_PREFETCH 2
+#endif
+constexpr int kVarPrefetch = LV_VAR_PREFETCH;  // grid columns between the L2 prefetch and the load
+
+// (bf16 pair) + (fp32 pair): the mixed-precision add converts its 16-bit operand exactly, so the
+// result is the fp32 sum rounded once, as with a separate conversion
+__device__ __forceinline__ float2 bf16x2_plus_f32x2(uint32_t w, float2 c) {
+  float2 r;
+  asm("{\n .reg .b16 lo, hi;\n mov.b32 {lo, hi}, %2;\n add.rn.f32.bf16 %0, lo, %3;\n add.rn.f32.bf16 %1, hi, %4;\n}"
+      : "=f"(r.x), "=f"(r.y)
+      : "r"(w), "f"(c.x), "f"(c.y));
+  return r;
+}
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 struct VarColumn {
   float2 s[kVarRows][4];  // vertical 3-sums of d, this lane's 8 channels as pairs (packed fp32 arithmetic)
@@ -170,7 +270,7 @@ __device__ __forceinline__ void var_column(const uint4 (&raw)[kVarRows + 2], con
     float2 q2 = make_float2(0.0f, 0.0f);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      d[r][i] = __fadd2_rn(make_float2(bf16_lo(w[i]), bf16_hi(w[i])), neg_x0[i]);
+      d[r][i] = bf16x2_plus_f32x2(w[i], neg_x0[i]);
       q2 = __ffma2_rn(d[r][i], d[r][i], q2);
     }
     q[r] = q2.x + q2.y;
@@ -243,6 +343,13 @@ var_map_kernel(const __nv_bfloat16* __restrict__ x, float* __restrict__ var, int
 #pragma unroll
       for (int r = 0; r < kVarRows + 2; ++r)
         if (row_ok[r]) raw[r] = __ldg(col_ptr + (ptrdiff_t)r * row_stride);
+    }
+    // the registers hold one column ahead; the columns after it are asked into L2 meanwhile, so
+    // the loads above find them there instead of waiting for HBM
+    if (c + kVarPrefetch < grid_w) {
+#pragma unroll
+      for (int r = 0; r < kVarRows + 2; ++r)
+        if (row_ok[r]) prefetch_l2(col_ptr + (ptrdiff_t)r * row_stride + kVarPrefetch * kVarTokenVec);
     }
   };
   // window of grid column px = columns a, b, c (an absent one is all-zero); `ab` = a + b
