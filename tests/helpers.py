@@ -80,7 +80,7 @@ def half_ulp_bf16(ref: np.ndarray) -> np.ndarray:
 
 
 def report(name: str, **values):
-    """Print one measured figure of a parity check and append it to gpurun_out/parity_report.jsonl
+    """Print one measured figure of a parity check and append it to the report file (_REPORT)
     (the tables of measured error against bound are made from that file)."""
     rec = {"check": name}
     rec.update({k: (float(v) if isinstance(v, (float, np.floating)) else v) for k, v in values.items()})

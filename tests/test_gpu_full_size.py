@@ -43,7 +43,11 @@ def run(request):
 
 
 def test_sizes_and_index_invariants(run):
-    ex, sz, ctx = run["ex"], run["sizes"], run["ctx"]
+    check_invariants(run, run["ex"])
+
+
+def check_invariants(run, ex):
+    sz, ctx = run["sizes"], run["ctx"]
     assert (ctx.n_tokens, ctx.n_merged, ctx.n_src, ctx.n_dst) == (sz["N"], sz["M"], sz["n_src"], sz["n_dst"])
     assert int(ex["size"].sum()) == sz["N"] and ex["size"].min() >= 1
     assert np.all(np.diff(ex["kept_idx"]) > 0)
@@ -58,21 +62,30 @@ def test_sizes_and_index_invariants(run):
     assert np.all(ex["cls"][owners] == O.CLS_DST)
 
 
-def test_grad_var_ga_maps_on_sampled_frames(run):
-    wl, ex = run["wl"], run["ex"]
+def check_maps_on_sampled_frames(run, ex, tokens):
+    """Grad map, Var map of `tokens` and GA map of the plan export `ex` on the sampled frames."""
+    wl = run["wl"]
     t = wl.tokens_per_frame
     grad_gpu = to_f64(run["grad"])
     for f in run["frames_sampled"]:
         ref_g = O.grad_map(run["images"][f:f + 1].cpu().numpy())[0]
         assert np.abs(grad_gpu[f] - ref_g).max() <= 1e-5 * max(ref_g.max(), 1e-3)
-        ref_v = O.var_map(to_f64(run["tokens"][f * t:(f + 1) * t]), 1, wl.grid_h, wl.grid_w)[0]
+        ref_v = O.var_map(to_f64(tokens[f * t:(f + 1) * t]), 1, wl.grid_h, wl.grid_w)[0]
         assert np.abs(ex["var"][f] - ref_v).max() <= 2e-5 * ref_v.max()
         ref_ga = O.ga_map(grad_gpu[f:f + 1], ex["var"][f:f + 1].astype(np.float64))[0]
         assert np.abs(ex["ga"][f] - ref_ga).max() <= 1e-5
 
 
+def test_grad_var_ga_maps_on_sampled_frames(run):
+    check_maps_on_sampled_frames(run, run["ex"], run["tokens"])
+
+
 def test_partition_counts_everywhere_and_classes_on_sampled_frames(run):
-    wl, ex, sz = run["wl"], run["ex"], run["sizes"]
+    check_partition(run, run["ex"])
+
+
+def check_partition(run, ex):
+    wl, sz = run["wl"], run["sizes"]
     per_frame = ex["cls"].reshape(wl.frames, wl.tokens_per_frame)
     assert np.all(per_frame[:, :5] == O.CLS_PROTECTED) and np.all(per_frame[0, 5:] == O.CLS_DST)
     rest = per_frame[1:, 5:]
@@ -102,12 +115,15 @@ N_MATCH_ROWS = 4096
 
 
 def test_matches_on_sampled_src_rows(run):
+    check_matches_on_sampled_src_rows(run, run["ex"], run["tokens"], run["wl"].name)
+
+
+def check_matches_on_sampled_src_rows(run, ex, tokens, tag):
     """4096 seeded src rows against every anchor of the sequence (the oracle's match on a compact
     copy: anchors first, then the sampled rows).  The stated tolerance in full: the argmax equals the
     oracle's wherever the oracle's top-1 / top-2 margin exceeds 1e-3, at least 99.9 % of the rows agree,
     and a row that differs is a near-tie (its similarity within 1e-5 of the oracle's best).  The margin
     histogram and the agreement are reported with the result."""
-    ex, tokens, wl = run["ex"], run["tokens"], run["wl"]
     src_idx = np.flatnonzero(ex["cls"] == O.CLS_SRC)
     dst_idx = np.flatnonzero(ex["cls"] == O.CLS_DST)
     rng = np.random.default_rng(5)
@@ -120,7 +136,7 @@ def test_matches_on_sampled_src_rows(run):
     best_token = dst_idx[best]
     margin = sim1 - sim2
     agree = ex["best_dst"][rows] == best_token
-    report(f"{wl.name}: matching on {rows.size} sampled src rows x {dst_idx.size} anchors",
+    report(f"{tag}: matching on {rows.size} sampled src rows x {dst_idx.size} anchors",
            agreement=float(agree.mean()), near_ties_accepted=int((~agree).sum()),
            margin_below_1e_5=float((margin < 1e-5).mean()), margin_below_1e_4=float((margin < 1e-4).mean()),
            margin_below_1e_3=float((margin < 1e-3).mean()), margin_median=float(np.median(margin)),
@@ -131,7 +147,11 @@ def test_matches_on_sampled_src_rows(run):
 
 
 def test_selection_and_index_arrays_bit_exact_given_the_matches(run):
-    ex, sz = run["ex"], run["sizes"]
+    check_index_arrays(run, run["ex"])
+
+
+def check_index_arrays(run, ex):
+    sz = run["sizes"]
     dst_of, size, kept = O.select_and_index(ex["cls"], ex["best_dst"], ex["best_sim"], sz["R"])
     assert np.array_equal(ex["dst_of"], dst_of)
     assert np.array_equal(ex["size"], size)
@@ -277,7 +297,8 @@ def test_block_sublayers_on_sampled_rows_and_frames(run):
 def test_qk_norm_and_rope_on_sampled_rows(run):
     """The optional Q/K normalisation and rotary embedding at full size: the transformed Q and K of
     sampled merged rows (first, last, tile edges, random) against the oracle on those rows, positions
-    taken from the owner tokens.  Runs last in this module: it overwrites the layer's intermediates."""
+    taken from the owner tokens.  Runs after the checks of the plain layer: it overwrites the layer's
+    intermediates."""
     ctx, xm, sz, wl, ex = run["ctx"], run["xm"], run["sizes"], run["wl"], run["ex"]
     w_qkv, b_qkv, w_o, b_o = run["weights"]
     gen = torch.Generator().manual_seed(wl.seed + 77)
@@ -303,6 +324,40 @@ def test_qk_norm_and_rope_on_sampled_rows(run):
     assert rel_err(got[:, 2048:], ref[:, 2048:]) <= bf16_bound(ref[:, 2048:]), "V is only projected"
     ref_y = O.linear(to_f64(ctx.debug_buffer(1)[rows_t]), to_f64(w_o), to_f64(b_o))
     assert rel_err(to_f64(y[rows_t]), ref_y) <= bf16_bound(ref_y), "output projection"
+
+
+def test_plan_refreshed_in_place_on_the_layer_output(run):
+    """Sec. 3.4, cached token merging at full size: the plan of the fixture is rebuilt IN PLACE (same
+    handle, its index arrays reused) on the features the layer has produced - the residual stream one
+    layer on, which is what a refresh layer of the schedule sees - and judged like the first build:
+    Var / GA maps and classes on sampled frames, matching on 4096 sampled src rows against all
+    anchors, selection and index arrays bit-exact given the matches, and the merge under the new plan
+    on sampled rows.  Last user of the fixture's plan."""
+    ctx, plan, wl, sz = run["ctx"], run["plan"], run["wl"], run["sizes"]
+    x2 = run["out"]
+    handle = plan.handle.value
+    assert ctx.merge_plan(x2, run["grad"], plan).handle.value == handle
+    xm2 = ctx.merge(plan, x2)
+    ctx.poll()
+    ex2 = ctx.plan_export(plan)
+    moved = float((ex2["dst_of"] != run["ex"]["dst_of"]).mean())
+    report(f"{wl.name}: plan refreshed in place on the layer output", tokens_with_another_row=moved,
+           classes_changed=float((ex2["cls"] != run["ex"]["cls"]).mean()))
+    assert moved > 0.0, "the refresh changed nothing: the drifted features were not used"
+    check_invariants(run, ex2)
+    check_maps_on_sampled_frames(run, ex2, x2)
+    check_partition(run, ex2)
+    check_matches_on_sampled_src_rows(run, ex2, x2, f"{wl.name} refreshed")
+    check_index_arrays(run, ex2)
+    order = np.argsort(ex2["dst_of"], kind="stable")
+    starts = np.concatenate([[0], np.cumsum(ex2["size"])])
+    rng = np.random.default_rng(16)
+    rows = np.unique(np.concatenate([rng.choice(sz["M"], 96, replace=False), np.argsort(ex2["size"])[-8:], [0, sz["M"] - 1]]))
+    ref = np.empty((rows.size, 1024))
+    for k, j in enumerate(rows):
+        members = order[starts[j]:starts[j + 1]]
+        ref[k] = to_f64(x2[torch.from_numpy(members).cuda()]).mean(axis=0)
+    check_bf16(f"{wl.name} refreshed: merge", to_f64(xm2[torch.from_numpy(rows).cuda()]), ref, sampled=True)
 
 
 @pytest.mark.parametrize("name", ["C3", "C5"])
