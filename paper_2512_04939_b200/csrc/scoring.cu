@@ -214,10 +214,11 @@ cudaError_t launch_grad_map(const litevggt_ctx* ctx, const float* images, float*
 // fully coalesced 512-byte load straight into registers, with no shared-memory stage and no
 // barrier.  The warp walks along the strip one grid column per step: the column's kVarRows + 2
 // tokens (one halo row above and below; outside the grid the lane's own x0 stands in, so d = 0)
-// are read once (the difference to x0 comes from a mixed-precision add that takes the bf16 value as
-// it is, so no separate conversion), give the column's vertical sums of d and of |d|^2, and the sums of the two
-// columns before stay in registers; the loads of the next column are issued as soon as this
-// column's registers are free.  A window's value, (1/n) sum |d|^2 - (1/n^2) |sum d|^2, is linear in
+// are read once (the difference to x0 comes from a mixed-precision add that takes the bf16 value
+// as it is, so there is no separate conversion) and give the column's vertical sums of d and of
+// |d|^2; the sums of the two columns before stay in registers; the loads of the next column are
+// issued as soon as this column's registers are free, and the column after it is asked into L2.
+// A window's value, (1/n) sum |d|^2 - (1/n^2) |sum d|^2, is linear in
 // the per-lane partial sums over the channels, so each lane forms it for its 8 channels, a
 // butterfly over the warp adds the 32 lanes for all rows of the strip at once, the four warps'
 // sums meet in shared memory and are added in a fixed order: the map is deterministic.
