@@ -302,8 +302,12 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       const uint32_t o_col = tmem_base + kFaColO + t * kFaOCols;
       const uint32_t q_col = tmem_base + kFaColQ + t * 32;
       // S_h = Q (tensor memory) x K[64h .. 64h+63]^T (shared memory, K-major); 4 steps of 16 channels
+      // the descriptors are linear in the shared-memory address (its 16-byte units sit in the low
+      // bits and cannot carry out of their field), so a stage / half is one addition away
+      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(smem_k), 16, 1024);
+      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(smem_v), kFaStages * kFaTileBytes, 1024);
       auto issue_qk = [&](int h, int stage) {
-        const uint64_t b_desc = smem_desc_sw128(smem_u32(smem_k + stage * kFaTileBytes + h * 8192), 16, 1024);
+        const uint64_t b_desc = k_desc0 + (uint64_t)((stage * kFaTileBytes + h * 8192) >> 4);
 #pragma unroll
         for (int k = 0; k < 4; ++k) umma_ts(s_col + h * 64, q_col + k * 8, b_desc + 2 * k, idesc_qk, k != 0 ? 1u : 0u);
         umma_commit(&bars->s_full[t][h]);
@@ -332,8 +336,7 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
           // 8 TMEM columns of P (keys 0-31 in columns [0,16) of the half, keys 32-63 in [32,48)),
           // 2048 bytes of V
           // second 64-column block of B = the ones block, one V ring further on
-          const uint64_t v_desc = smem_desc_sw128(smem_u32(smem_v + stage * kFaTileBytes + h * 8192),
-                                                  kFaStages * kFaTileBytes, 1024);
+          const uint64_t v_desc = v_desc0 + (uint64_t)((stage * kFaTileBytes + h * 8192) >> 4);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             umma_ts(o_col, s_col + h * 64 + (k >> 1) * 32 + (k & 1) * 8, v_desc + 128 * k, idesc_pv,
@@ -419,16 +422,18 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
       // they come out of the tensor core.
       m_ref = 0.0f;
       pair_syncs = n_steps;  // this form has no pair barriers
-      for (int n = 0; n < n_steps; ++n) {
-        const int j = n >> 1, h = n & 1;
-        if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
+      // One step = this thread's 32 scores of one half of a key tile.  Only the last tile of a
+      // launch can reach past the sequence, so the steps before it need no masking; the two halves
+      // are written out so that barrier and tensor-memory addresses are constants of the loop.
+      auto step = [&](int j, int h, bool may_mask) -> bool {
+        if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) return false;
         tc_fence_after();
         uint32_t s[32];
         tmem_ld32(s_addr + h * 64 + c * 32, s);
         tmem_ld_wait();
-        const int valid = seq_len - (tile_begin * 2 + n) * 64 - c * 32;
         uint32_t packed[16];
-        if (valid < 32) {
+        const int valid = may_mask ? seq_len - ((tile_begin + j) * 2 + h) * 64 - c * 32 : 32;
+        if (may_mask && valid < 32) {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
             if (i >= valid) s[i] = 0xff800000u;  // -inf: probability 0 (the polynomial cannot take it)
@@ -441,7 +446,10 @@ flash_attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __nv_
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
-      }
+        return true;
+      };
+      for (int j = 0; j + 1 < n_kv && ok; ++j) ok = step(j, 0, false) && step(j, 1, false);
+      if (ok && n_kv > 0) ok = step(n_kv - 1, 0, true) && step(n_kv - 1, 1, true);
     } else {
     // ---- online form
     for (int n = 0; n < n_steps; ++n) {
