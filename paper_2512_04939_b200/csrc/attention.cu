@@ -801,18 +801,21 @@ flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __
     float m_ref = -INFINITY;
     bool ok = true;
     int pair_syncs = 0;
-    for (int n = 0; n < n_steps; ++n) {
-      const int j = n >> 1, h = n & 1;
-      if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) { ok = false; break; }
+    // the two halves of a key tile are written out (barrier and tensor-memory addresses constant);
+    // only the last tile of a launch can reach past the sequence
+    auto step = [&](int j, int h, bool may_mask) -> bool {
+      if (!mbar_wait_warp(&bars->s_full[t][h], j & 1, ctl)) return false;
       tc_fence_after();
       uint32_t s[32];
       tmem_ld32(s_addr + h * 64 + c * 32, s);
       tmem_ld_wait();
-      const int valid = seq_len - (tile_begin * 2 + n) * 64 - c * 32;
-      if (valid < 32) {
+      if (may_mask) {
+        const int valid = seq_len - ((tile_begin + j) * 2 + h) * 64 - c * 32;
+        if (valid < 32) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i >= valid) s[i] = 0xff800000u;  // -inf
+          for (int i = 0; i < 32; ++i)
+            if (i >= valid) s[i] = 0xff800000u;  // -inf
+        }
       }
       float mx[4];
 #pragma unroll
@@ -824,11 +827,11 @@ flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __
         mx[g] = fmaxf(mx[g], __uint_as_float(sc[7]));
       }
       const float mx_own = fmaxf(fmax3(mx[0], mx[1], mx[2]), mx[3]);
-      xchg->row_max[n & 1][t][c][row_in_tile] = mx_own;
+      xchg->row_max[h][t][c][row_in_tile] = mx_own;
       pair_barrier(barrier_id);
       ++pair_syncs;
-      const float mx_scaled = fmaxf(mx_own, xchg->row_max[n & 1][t][c ^ 1][row_in_tile]) * scale_log2e;
-      if (n == 0) {
+      const float mx_scaled = fmaxf(mx_own, xchg->row_max[h][t][c ^ 1][row_in_tile]) * scale_log2e;
+      if ((j | h) == 0) {
         m_ref = mx_scaled - kFa8Headroom;
       } else {
         const bool grow = mx_scaled > m_ref + kFa8Headroom + 0.75f;
@@ -837,7 +840,7 @@ flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __
           const bool waited = jp + 1 < n_kv
                                   ? mbar_wait_warp(&bars->s_full[t][h ^ 1], (uint32_t)(jp + 1) & 1u, ctl)
                                   : mbar_wait_warp(&bars->pv_done[t], 0, ctl);
-          if (!waited) { ok = false; break; }
+          if (!waited) return false;
           tc_fence_after();
           const float m_new = grow ? mx_scaled - kFa8Headroom : m_ref;
           const float alpha = fast_exp2(m_ref - m_new);
@@ -870,7 +873,10 @@ flash_attention_fp8_kernel(const __grid_constant__ CUtensorMap tmap_k8, const __
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_ready[t][h]);
-    }
+      return true;
+    };
+    for (int j = 0; j + 1 < n_kv && ok; ++j) ok = step(j, 0, false) && step(j, 1, false);
+    if (ok && n_kv > 0) ok = step(n_kv - 1, 0, true) && step(n_kv - 1, 1, true);
     for (; pair_syncs < n_steps; ++pair_syncs) pair_barrier(barrier_id);
     if (ok && mbar_wait_warp(&bars->o_done[t], 0, ctl)) {
       tc_fence_after();
