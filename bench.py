@@ -40,7 +40,7 @@ METRIC = "frames/s through merge+global-attn+unmerge (plan refreshed every 6th l
 # workload C5, summed over the layer's key-chunk launches, from one single-pass ncu capture
 # (profiles/flash_attention_C5_dram.md).  Reported only while the kernel source is the one that was
 # measured.
-ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 34.64e9 + 17.61e9, "kernel_sha256": "b9b804506460376a54d9d266dd3466072b2e64d8a413a42bf9fc51279a195271"}
+ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 34.63e9 + 17.60e9, "kernel_sha256": "14bea7adbb74f9b3ba9530f578778ce40e8cac4d59aec3e64d1f581c18d6e78f"}
 
 
 def _attention_source_hash() -> str:
