@@ -87,10 +87,12 @@ constexpr int kFaTileBytes = 128 * 64 * 2;
 constexpr uint32_t kFaColS = 0, kFaColO = 256, kFaColQ = 416;
 constexpr uint32_t kFaOCols = 80;  // 64 output channels, the row sum, 15 unused columns
 constexpr float kFaRescaleThreshold = 8.0f;
-// Largest Cauchy-Schwarz bound on the base-2 scores of a row for which the fixed reference is
-// used: probabilities go down to 2^-96, their products with |v| >= 2^-20 stay normal in fp32.
+// Largest Cauchy-Schwarz bound B on the base-2 scores of a row for which the fixed reference is
+// used.  With the reference left out the probabilities lie in [2^-B, 2^B]: at B = 80 their products
+// with |v| >= 2^-20 are normal fp32 numbers (>= 2^-100), and a row sum over 2^20 keys times
+// |v| <= 2^20 stays below 2^120, inside fp32; the polynomial exponential is valid to +-120.
 #ifndef LV_FA_FIXED_REF_LIMIT
-#define LV_FA_FIXED_REF_LIMIT 48.0f
+#define LV_FA_FIXED_REF_LIMIT 80.0f
 #endif
 constexpr float kFaFixedRefLimit = LV_FA_FIXED_REF_LIMIT;
 #ifndef LV_FA_CHUNK_TILES
@@ -98,7 +100,7 @@ constexpr float kFaFixedRefLimit = LV_FA_FIXED_REF_LIMIT;
 #endif
 constexpr int kFaChunkTiles = LV_FA_CHUNK_TILES;  // 65536 keys: K and V of one head = 16 MiB
 // Of the 16 pairs of scores a thread handles per step, this many take the polynomial exponential
-// (fixed-reference form only, where every argument lies in [-2 * kFaFixedRefLimit, 0]).
+// (fixed-reference form only, where every argument lies in [-kFaFixedRefLimit, kFaFixedRefLimit]).
 #ifndef LV_FA_POLY_PAIRS
 #define LV_FA_POLY_PAIRS 7
 #endif

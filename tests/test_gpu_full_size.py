@@ -218,21 +218,25 @@ def key_chunk_edges(m):
     return [c * per_chunk * 128 for c in range(1, n_chunks)], per_chunk * 128
 
 
-@pytest.mark.parametrize("name", ["C3", "C4", "C5"])
-def test_attention_core_with_peaked_softmax_across_key_chunks(name):
+@pytest.mark.parametrize("name,sharpness", [("C3", 4.0), ("C4", 4.0), ("C5", 4.0), ("C3", 16.0), ("C5", 16.0)])
+def test_attention_core_with_peaked_softmax_across_key_chunks(name, sharpness):
     """The attention core at the merged lengths of C3, C4 and C5 on inputs whose softmax is far from
     uniform: every query's mass sits on itself and on the ~M/4099 rows of its group, which lie 4099
     rows apart through the whole sequence, so every key chunk (C3: 2, C4: 4, C5: 8) carries a share of every
     output.  Sampled queries sit on both sides of every chunk boundary, at tile edges and at random.
-    A chunk left out on the oracle's side must move the result far beyond the tolerance."""
+    A chunk left out on the oracle's side must move the result far beyond the tolerance.
+    Sharpness 4 keeps every row's score bound under the limit of the fixed softmax reference;
+    sharpness 16 puts them over it, so the running-maximum form and its combination of chunks with
+    different references are the ones under test."""
     import paper_2512_04939_b200 as pkg
 
     wl = WORKLOADS[name]
     ctx = pkg.LiteVGGT(wl.frames, wl.grid_h, wl.grid_w, wl.merge_ratio)
     m = ctx.n_merged
-    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, wl.seed + 9, "cuda")
+    x, w_qkv, b_qkv, w_o, b_o = make_peaked_attention_inputs(m, wl.seed + 9, "cuda", sharpness=sharpness)
     ctx.global_attn(x, w_qkv, b_qkv, w_o, b_o)
     ctx.poll()
+    name = f"{name}, sharpness {sharpness:g}"
     edges, chunk_rows = key_chunk_edges(m)
     rng = np.random.default_rng(17)
     rows = [0, 127, 128, 255, 256, m - 129, m - 128, m - 1] + list(rng.choice(m, 16, replace=False))

@@ -331,7 +331,7 @@ def score_bounds(qkv, heads=16):
     return np.sqrt((q * q).sum(-1)) * np.sqrt((k * k).sum(-1)).max(0)
 
 
-FIXED_REF_LIMIT = 48.0  # the library's kFaFixedRefLimit
+FIXED_REF_LIMIT = 80.0  # the library's kFaFixedRefLimit
 
 
 @pytest.mark.parametrize("wl", [WORKLOADS["C1"], MID], ids=lambda w: w.name)
@@ -341,13 +341,13 @@ def test_global_attention(lib, wl):
     m = ref["sizes"]["M"]
     xm = torch.from_numpy(O.merge(to_f64(tok), ref["dst_of"], m).astype(np.float32)).to(torch.bfloat16)
     w_qkv, b_qkv, w_o, b_o = make_attention_weights(wl, 0)
-    # second pass with 3x larger projection weights: the softmax becomes far from uniform
+    # second pass with 4x larger projection weights: the softmax becomes far from uniform
     # (random-init 0.02 weights alone give nearly flat attention, which would hide
     # indexing mistakes) and the score bound of most rows passes the limit of the
     # fixed-reference form, so the online form runs
-    w_big = (w_qkv.float() * 3.0).to(torch.bfloat16)
+    w_big = (w_qkv.float() * 4.0).to(torch.bfloat16)
     ctx = _ctx(lib, wl)
-    for tag, wq in (("stock", w_qkv), ("3x", w_big)):
+    for tag, wq in (("stock", w_qkv), ("4x", w_big)):
         y = ctx.global_attn(xm.cuda(), wq.cuda(), b_qkv.cuda(), w_o.cuda(), b_o.cuda())
         ctx.poll()
         # each stage against the oracle fed with the GPU's own upstream (bf16) result
@@ -371,12 +371,13 @@ def test_global_attention(lib, wl):
     ctx.close()
 
 
-@pytest.mark.parametrize("grid,sharpness,form", [((22, 33), 4.0, "fixed"), ((22, 33), 8.0, "online"),
+@pytest.mark.parametrize("grid,sharpness,form", [((22, 33), 4.0, "fixed"), ((22, 33), 6.0, "fixed"), ((22, 33), 16.0, "online"),
                                                  ((34, 44), 4.0, "fixed")])
 def test_attention_core_with_peaked_softmax(lib, grid, sharpness, form):
     """Rows in groups of near-duplicates spread through the sequence and query weights a multiple of
     the key weights: a row's probability mass sits on itself and its group, so every key tile
-    matters.  sharpness 4 keeps the score bounds under the fixed-reference limit, 8 puts them over."""
+    matters.  sharpness 4 and 6 keep the score bounds under the fixed-reference limit (6: up to 70, the upper
+    part of what that form takes), 16 puts them over."""
     ctx = lib.LiteVGGT(2, grid[0], grid[1], 0.0)  # merge ratio 0: M = N (1462 / 3002 rows, ragged tiles)
     m = ctx.n_merged
     assert m == ctx.n_tokens
