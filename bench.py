@@ -40,7 +40,7 @@ METRIC = "frames/s through merge+global-attn+unmerge (plan refreshed every 6th l
 # workload C5, summed over the layer's key-chunk launches, from one single-pass ncu capture
 # (profiles/flash_attention_C5_dram.md).  Reported only while the kernel source is the one that was
 # measured.
-ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 34.63e9 + 17.60e9, "kernel_sha256": "14bea7adbb74f9b3ba9530f578778ce40e8cac4d59aec3e64d1f581c18d6e78f"}
+ATTENTION_TRAFFIC_C5 = {"bytes_per_layer": 34.65e9 + 17.60e9, "kernel_sha256": "dce9e561e33d972a66c4798f3eb9686614976653cbcabe9afecc16fd9265da67"}
 
 
 def _attention_source_hash() -> str:
